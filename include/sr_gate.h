@@ -1,0 +1,169 @@
+/*
+ * sr_gate.h -- C ABI of the Selective Rollout gate library (NVIDIA B200, sm_100a).
+ *
+ * The library evaluates, for many GRPO groups at once, the gate of the paper's
+ * Section 3.2: the mean pairwise prefix edit distance d_K between the N partial
+ * action sequences of a group, the decision Cut = [d_K < d_L] (Eq. 2), and the
+ * group-relative advantages of Eq. 1 with the zero-variance flag of Section 2.1.
+ *
+ * Conventions (every entry point unless it says otherwise)
+ *   - Pointers are DEVICE pointers.  The caller owns every buffer; the library
+ *     allocates no device memory and keeps no state between calls.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work on it and return without synchronising.
+ *   - Return value: SR_OK, or a negative SR_ERR_* code, in which case nothing was
+ *     enqueued and no buffer was touched.
+ *   - Actions (or tokens) are int32 IDs compared for equality only; every 32-bit
+ *     value is legal.  Mapping action strings to IDs is the caller's job.
+ *   - Pairs of a group are ordered (0,1),(0,2),...,(0,N-1),(1,2),...,(N-2,N-1);
+ *     P = N(N-1)/2.
+ */
+#ifndef SR_GATE_H_
+#define SR_GATE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SR_VERSION 100
+
+/* error codes */
+#define SR_OK 0
+#define SR_ERR_NULL (-1)           /* a required pointer is NULL */
+#define SR_ERR_BAD_N (-2)          /* N < 2 or N > SR_MAX_N, or n_groups < 0 */
+#define SR_ERR_BAD_K (-3)          /* K < 0, K > stride, K > SR_MAX_K, bad max_steps */
+#define SR_ERR_ALIGN (-4)          /* seqs not 16-byte aligned or stride % 4 != 0 */
+#define SR_ERR_STATE_SIZE (-5)     /* incremental state buffer too small */
+#define SR_ERR_WORKSPACE (-6)      /* workspace NULL, misaligned or too small */
+#define SR_ERR_CUDA (-7)           /* a CUDA call failed; see sr_last_cuda_error() */
+#define SR_ERR_BAD_MODE (-8)       /* unknown norm_mode */
+
+/* limits */
+#define SR_MAX_N 32                /* rollouts per group */
+#define SR_MAX_K 1024              /* longest prefix (symbols) */
+#define SR_MAX_INCR_STEPS 32       /* longest rollout the incremental state can hold */
+
+/* norm_mode */
+#define SR_NORM_MAXLEN 0           /* paper: each pair distance / longer prefix length */
+#define SR_NORM_NONE 1             /* mean of the raw pair distances */
+
+/* new_actions value meaning "this rollout emitted no action this step" */
+#define SR_NO_ACTION INT32_MIN
+
+/* bits OR-ed into *status by the kernels (the caller zeroes it when it wants to) */
+#define SR_STATUS_NEG_LEN 1        /* a negative length was treated as 0 */
+#define SR_STATUS_STEP_OVERFLOW 2  /* an action arrived for a rollout already at max_steps; ignored */
+#define SR_STATUS_BAD_STATE 4      /* incremental state header does not match the call; step skipped */
+
+int sr_version(void);
+const char* sr_strerror(int code);      /* static string */
+const char* sr_last_cuda_error(void);   /* text of the last CUDA failure seen by this thread */
+
+/*
+ * sr_gate -- d_K and the stop mask for every group (Section 3.2, Appendix B
+ * "prefix_edit_distance_mean", Eq. 2).
+ *
+ * For each group g and each pair i<j: d_ij = unit-cost Levenshtein distance
+ * (insert / delete / substitute) between the first m_i = min(len_i, K) IDs of
+ * rollout i and the first m_j of rollout j.  With SR_NORM_MAXLEN each d_ij is
+ * divided by max(m_i, m_j) (0 when both prefixes are empty); the terms are added
+ * in fp64 in pair order and divided by P, giving mean[g] = d_K.  stop[g] =
+ * (mean[g] < threshold), strictly.  Negative lengths count as 0 and set
+ * SR_STATUS_NEG_LEN.
+ *
+ *   seqs       in  [n_groups][N][stride] int32, row-major, 16-byte aligned, stride % 4 == 0
+ *   lens       in  [n_groups][N] int32 actions emitted so far; NULL = every length is K
+ *   K              gate step, 0 <= K <= min(stride, SR_MAX_K)
+ *   threshold      d_L
+ *   pair_dist  out [n_groups][P] int32 raw distances; may be NULL
+ *   pair_sum   out [n_groups] int32 sum of the raw distances; may be NULL
+ *   mean       out [n_groups] fp64; may be NULL
+ *   stop       out [n_groups] uint8, 1 = cut; required
+ *   status     in/out 1 int32 of SR_STATUS_* bits; may be NULL
+ *   workspace      device scratch of at least sr_gate_workspace_bytes(...) bytes,
+ *                  256-byte aligned; contents are undefined before and after the
+ *                  call; may be NULL when that size is 0 (K <= 32).  Two calls
+ *                  that may overlap on the device need separate workspaces.
+ *
+ * n_groups == 0 is a valid no-op.  Prefixes of up to 32 symbols use one 32-bit
+ * word of bit-parallel state per pair; longer ones use the blocked multi-word path.
+ */
+int sr_gate(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+            int32_t stride, int32_t K, double threshold, int32_t norm_mode,
+            int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+            int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Host-only, pure.  Scratch bytes sr_gate needs for these sizes (0 when K <= 32);
+ * returns 0 for invalid arguments as well (sr_gate then reports the error). */
+size_t sr_gate_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
+
+/*
+ * sr_gate_host -- the same computation on HOST buffers: copies seqs/lens to the
+ * device, runs sr_gate, and copies the requested outputs back, all enqueued on
+ * `stream`; the caller synchronises the stream before reading the outputs.
+ * Every data pointer here is a HOST pointer (pinned memory makes the copies
+ * asynchronous); outputs that are NULL are not copied.  `arena` is DEVICE scratch
+ * of at least sr_gate_host_arena_bytes(...) bytes, 256-byte aligned, used for the
+ * staged inputs, outputs and the gate workspace.
+ */
+int sr_gate_host(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                 int32_t stride, int32_t K, double threshold, int32_t norm_mode,
+                 int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                 int32_t* status, void* arena, size_t arena_bytes, void* stream);
+size_t sr_gate_host_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
+
+/*
+ * Incremental gate: the gate re-evaluated after every environment step while
+ * each rollout appends one action per step.  The paper evaluates the gate at one
+ * fixed step K (Appendix C.1) and names an adaptive K as future work (Section 5,
+ * Limitations); this variant keeps, per pair, the boundary of the edit-distance
+ * matrix (vertical deltas of the last column, horizontal deltas of the last row,
+ * as +1 / -1 bit masks) in a caller-owned device buffer, so one step costs a
+ * constant number of word operations per pair.  After every step the outputs
+ * equal sr_gate(K = max_steps) on the prefixes emitted so far.
+ *
+ * The state is position independent: a byte copy of the buffer is a valid
+ * snapshot and can be restored into any other buffer of the same size.
+ *
+ *   sr_incr_state_bytes  host-only, pure; 0 for invalid arguments
+ *   sr_incr_init         formats `state` for n_groups x N rollouts of length 0;
+ *                        max_steps in 1..SR_MAX_INCR_STEPS
+ *   sr_gate_step_incremental
+ *     new_actions in  [n_groups][N] int32; SR_NO_ACTION = no action this step.
+ *                     An action for a rollout already holding max_steps actions is
+ *                     ignored and sets SR_STATUS_STEP_OVERFLOW.
+ *     outputs as for sr_gate (pair_dist, pair_sum, mean may be NULL).
+ *     n_groups, N must match sr_incr_init, else SR_STATUS_BAD_STATE is set and
+ *     the step does nothing.
+ */
+size_t sr_incr_state_bytes(int32_t n_groups, int32_t N, int32_t max_steps);
+int sr_incr_init(void* state, size_t state_bytes, int32_t n_groups, int32_t N,
+                 int32_t max_steps, void* stream);
+int sr_gate_step_incremental(void* state, size_t state_bytes, const int32_t* new_actions,
+                             int32_t n_groups, int32_t N, double threshold, int32_t norm_mode,
+                             int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                             int32_t* status, void* stream);
+
+/*
+ * sr_grpo_advantage -- Eq. 1: A_i = (r_i - mean_r) / (sigma_r + eps) with the
+ * population standard deviation (1/N), accumulated in fp64 and rounded once to
+ * fp32.  zero_var[g] = 1 iff all N rewards of the group compare equal (Section
+ * 2.1); such a group, and every group whose drop_mask byte is non-zero (a group
+ * cut by the gate never enters the loss, Appendix C.1), gets A_i = +0.0 exactly.
+ * NaN rewards compare unequal and propagate.
+ *
+ *   rewards    in  [n_groups][N] fp32
+ *   drop_mask  in  [n_groups] uint8 or NULL
+ *   adv        out [n_groups][N] fp32
+ *   zero_var   out [n_groups] uint8; may be NULL
+ */
+int sr_grpo_advantage(const float* rewards, const uint8_t* drop_mask, int32_t n_groups,
+                      int32_t N, float eps, float* adv, uint8_t* zero_var, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SR_GATE_H_ */

@@ -1,0 +1,187 @@
+"""Thin ctypes binding of the sr_gate C ABI (include/sr_gate.h, include/sr_probe.h).
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+PyTorch tensors are used as device (or pinned host) memory and for streams.  There
+is no CPU fallback: if the shared library is missing or fails to load, every call
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libsr_gate.so")
+
+SR_OK = 0
+SR_ERR_NULL, SR_ERR_BAD_N, SR_ERR_BAD_K, SR_ERR_ALIGN = -1, -2, -3, -4
+SR_ERR_STATE_SIZE, SR_ERR_WORKSPACE, SR_ERR_CUDA, SR_ERR_BAD_MODE = -5, -6, -7, -8
+SR_NORM_MAXLEN, SR_NORM_NONE = 0, 1
+SR_NO_ACTION = -(2 ** 31)
+SR_STATUS_NEG_LEN, SR_STATUS_STEP_OVERFLOW, SR_STATUS_BAD_STATE = 1, 2, 4
+SR_MAX_N, SR_MAX_K, SR_MAX_INCR_STEPS = 32, 1024, 32
+SR_PROBE_LOGIC, SR_PROBE_ADD, SR_PROBE_MIX = 0, 1, 2
+
+_vp, _i32, _f64, _f32, _sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_double, ctypes.c_float, ctypes.c_size_t
+
+_SIGNATURES = {
+    "sr_version": (ctypes.c_int, []),
+    "sr_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+    "sr_last_cuda_error": (ctypes.c_char_p, []),
+    "sr_gate": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp, _vp,
+                               _vp, _sz, _vp]),
+    "sr_gate_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
+    "sr_gate_host": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
+                                    _vp, _vp, _sz, _vp]),
+    "sr_gate_host_arena_bytes": (_sz, [_i32, _i32, _i32, _i32]),
+    "sr_incr_state_bytes": (_sz, [_i32, _i32, _i32]),
+    "sr_incr_init": (ctypes.c_int, [_vp, _sz, _i32, _i32, _i32, _vp]),
+    "sr_gate_step_incremental": (ctypes.c_int, [_vp, _sz, _vp, _i32, _i32, _f64, _i32, _vp, _vp, _vp,
+                                                _vp, _vp, _vp]),
+    "sr_grpo_advantage": (ctypes.c_int, [_vp, _vp, _i32, _i32, _f32, _vp, _vp, _vp]),
+    "sr_probe_int32": (ctypes.c_int, [_i32, _i32, _i32, _i32, _vp, _vp]),
+    "sr_probe_int32_ops": (ctypes.c_uint64, [_i32, _i32, _i32]),
+}
+
+_lib = None
+
+
+class SrError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(what)
+
+
+def load() -> ctypes.CDLL:
+    """Load libsr_gate.so (built in-tree by ``python -m paper_2605_05802_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise SrError(SR_ERR_CUDA, f"{LIB_PATH} is missing: build it with "
+                                       "`python -m paper_2605_05802_b200.build`; there is no fallback path")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != SR_OK:
+        lib = load()
+        msg = lib.sr_strerror(rc).decode()
+        if rc == SR_ERR_CUDA:
+            msg += ": " + lib.sr_last_cuda_error().decode()
+        raise SrError(rc, f"sr_gate error {rc}: {msg}")
+
+
+def _ptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype] = None) -> Optional[int]:
+    if t is None:
+        return None
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def sr_version() -> int:
+    return int(load().sr_version())
+
+
+def sr_strerror(code: int) -> str:
+    return load().sr_strerror(code).decode()
+
+
+def sr_gate_workspace_bytes(n_groups: int, N: int, stride: int, K: int) -> int:
+    return int(load().sr_gate_workspace_bytes(n_groups, N, stride, K))
+
+
+def sr_gate(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, threshold: float,
+            norm_mode: int = SR_NORM_MAXLEN, *, pair_dist: Optional[torch.Tensor] = None,
+            pair_sum: Optional[torch.Tensor] = None, mean: Optional[torch.Tensor] = None,
+            stop: torch.Tensor = None, status: Optional[torch.Tensor] = None,
+            workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    """seqs int32 [G, N, stride] on the device; outputs are preallocated tensors."""
+    G, N, stride = seqs.shape
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().sr_gate(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
+                          float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
+                          _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
+                          _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(workspace),
+                          ws_bytes, _stream(stream)))
+
+
+def sr_gate_host_arena_bytes(n_groups: int, N: int, stride: int, K: int) -> int:
+    return int(load().sr_gate_host_arena_bytes(n_groups, N, stride, K))
+
+
+def sr_gate_host(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, threshold: float,
+                 norm_mode: int = SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None, mean=None,
+                 stop=None, status=None, arena: torch.Tensor = None, stream=None) -> None:
+    """Same as sr_gate with HOST tensors (ideally pinned) for inputs and outputs and
+    a device ``arena``; the caller synchronises the stream before reading outputs."""
+    for t in (seqs, lens, pair_dist, pair_sum, mean, stop, status):
+        if t is not None and t.is_cuda:
+            raise ValueError("sr_gate_host takes host tensors")
+    G, N, stride = seqs.shape
+    _check(load().sr_gate_host(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
+                               float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
+                               _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
+                               _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(arena),
+                               arena.numel() * arena.element_size(), _stream(stream)))
+
+
+def sr_incr_state_bytes(n_groups: int, N: int, max_steps: int) -> int:
+    return int(load().sr_incr_state_bytes(n_groups, N, max_steps))
+
+
+def sr_incr_init(state: torch.Tensor, n_groups: int, N: int, max_steps: int, stream=None) -> None:
+    _check(load().sr_incr_init(_ptr(state), state.numel() * state.element_size(), n_groups, N,
+                               max_steps, _stream(stream)))
+
+
+def sr_gate_step_incremental(state: torch.Tensor, new_actions: torch.Tensor, threshold: float,
+                             norm_mode: int = SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None,
+                             mean=None, stop=None, status=None, stream=None) -> None:
+    G, N = new_actions.shape
+    _check(load().sr_gate_step_incremental(
+        _ptr(state), state.numel() * state.element_size(), _ptr(new_actions, torch.int32), G, N,
+        float(threshold), norm_mode, _ptr(pair_dist, torch.int32), _ptr(pair_sum, torch.int32),
+        _ptr(mean, torch.float64), _ptr(stop, torch.uint8), _ptr(status, torch.int32),
+        _stream(stream)))
+
+
+def sr_grpo_advantage(rewards: torch.Tensor, drop_mask: Optional[torch.Tensor], eps: float, *,
+                      adv: torch.Tensor, zero_var: Optional[torch.Tensor] = None, stream=None) -> None:
+    G, N = rewards.shape
+    _check(load().sr_grpo_advantage(_ptr(rewards, torch.float32), _ptr(drop_mask, torch.uint8), G, N,
+                                    float(eps), _ptr(adv, torch.float32), _ptr(zero_var, torch.uint8),
+                                    _stream(stream)))
+
+
+def sr_probe_int32(variant: int, iters: int, blocks: int, threads: int, sink: torch.Tensor,
+                   stream=None) -> None:
+    _check(load().sr_probe_int32(variant, iters, blocks, threads, _ptr(sink), _stream(stream)))
+
+
+def sr_probe_int32_ops(iters: int, blocks: int, threads: int) -> int:
+    return int(load().sr_probe_int32_ops(iters, blocks, threads))
+
+
+def shard_groups(n_groups: int, world_size: int, rank: int):
+    """Contiguous range of groups owned by ``rank``: groups are independent (each
+    rollout worker applies the gate to its own groups, Appendix C.1), so sharding
+    needs no exchange."""
+    base, extra = divmod(n_groups, world_size)
+    lo = rank * base + min(rank, extra)
+    return lo, lo + base + (1 if rank < extra else 0)

@@ -1,0 +1,186 @@
+// extern "C" boundary of the sr_gate library: argument validation and dispatch.
+// Every check runs on the host before anything is enqueued, so an error return
+// guarantees that no buffer was touched.
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace sr {
+
+static thread_local char g_cuda_error[256] = "no CUDA error recorded";
+
+void note_cuda_error(cudaError_t e, const char* where) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s (%s)", where, cudaGetErrorName(e),
+             cudaGetErrorString(e));
+}
+
+static int check_gate_args(const int32_t* seqs, int32_t n_groups, int32_t N, int32_t stride,
+                           int32_t K, int32_t norm_mode, const uint8_t* stop) {
+    if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;
+    if (stride < 0 || K < 0 || K > stride || K > SR_MAX_K) return SR_ERR_BAD_K;
+    if (norm_mode != SR_NORM_MAXLEN && norm_mode != SR_NORM_NONE) return SR_ERR_BAD_MODE;
+    if (n_groups > 0 && (seqs == nullptr || stop == nullptr)) return SR_ERR_NULL;
+    if ((stride & 3) != 0 || (reinterpret_cast<uintptr_t>(seqs) & 15) != 0) return SR_ERR_ALIGN;
+    return SR_OK;
+}
+
+struct HostArena {
+    size_t off_seqs, off_lens, off_dist, off_sum, off_mean, off_stop, off_status, off_ws, total;
+};
+
+static HostArena host_arena(int32_t n_groups, int32_t N, int32_t stride, int32_t K) {
+    HostArena h;
+    const size_t P = pairs_of(N);
+    size_t off = 0;
+    h.off_seqs = off;   off = align_up(off + (size_t)n_groups * N * stride * 4, 256);
+    h.off_lens = off;   off = align_up(off + (size_t)n_groups * N * 4, 256);
+    h.off_dist = off;   off = align_up(off + (size_t)n_groups * P * 4, 256);
+    h.off_sum = off;    off = align_up(off + (size_t)n_groups * 4, 256);
+    h.off_mean = off;   off = align_up(off + (size_t)n_groups * 8, 256);
+    h.off_stop = off;   off = align_up(off + (size_t)n_groups, 256);
+    h.off_status = off; off = align_up(off + 4, 256);
+    h.off_ws = off;     off += sr_gate_workspace_bytes(n_groups, N, stride, K);
+    h.total = align_up(off, 256);
+    return h;
+}
+
+}  // namespace sr
+
+using namespace sr;
+
+extern "C" {
+
+int sr_version(void) { return SR_VERSION; }
+
+const char* sr_strerror(int code) {
+    switch (code) {
+        case SR_OK: return "ok";
+        case SR_ERR_NULL: return "a required pointer is NULL";
+        case SR_ERR_BAD_N: return "N outside 2..32 or negative group count";
+        case SR_ERR_BAD_K: return "K / stride / max_steps out of range";
+        case SR_ERR_ALIGN: return "seqs must be 16-byte aligned and stride a multiple of 4";
+        case SR_ERR_STATE_SIZE: return "incremental state buffer too small";
+        case SR_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case SR_ERR_CUDA: return "a CUDA call failed (see sr_last_cuda_error)";
+        case SR_ERR_BAD_MODE: return "unknown norm_mode";
+        default: return "unknown error code";
+    }
+}
+
+const char* sr_last_cuda_error(void) { return g_cuda_error; }
+
+size_t sr_gate_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K) {
+    if (n_groups < 0 || N < 2 || N > SR_MAX_N || K < 0 || K > stride || K > SR_MAX_K) return 0;
+    if (K <= 32) return 0;
+    return gate_multi_workspace_bytes(n_groups, N, stride, K);
+}
+
+int sr_gate(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N, int32_t stride,
+            int32_t K, double threshold, int32_t norm_mode, int32_t* pair_dist, int32_t* pair_sum,
+            double* mean, uint8_t* stop, int32_t* status, void* workspace, size_t workspace_bytes,
+            void* stream) {
+    const int rc = check_gate_args(seqs, n_groups, N, stride, K, norm_mode, stop);
+    if (rc != SR_OK) return rc;
+    GateArgs a{seqs, lens, n_groups, N, stride, K, threshold, norm_mode,
+               pair_dist, pair_sum, mean, stop, status};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (K <= 32) return launch_gate_single(a, s);
+    if (n_groups > 0) {
+        const size_t need = gate_multi_workspace_bytes(n_groups, N, stride, K);
+        if (workspace == nullptr || workspace_bytes < need ||
+            (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
+            return SR_ERR_WORKSPACE;
+    }
+    return launch_gate_multi(a, workspace, workspace_bytes, s);
+}
+
+size_t sr_gate_host_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K) {
+    if (n_groups < 0 || N < 2 || N > SR_MAX_N || stride < 0 || K < 0 || K > stride || K > SR_MAX_K)
+        return 0;
+    return host_arena(n_groups, N, stride, K).total;
+}
+
+int sr_gate_host(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                 int32_t stride, int32_t K, double threshold, int32_t norm_mode,
+                 int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                 int32_t* status, void* arena, size_t arena_bytes, void* stream) {
+    // the alignment rule applies to the device copy, which the arena guarantees
+    const int32_t* aligned_stand_in = seqs ? reinterpret_cast<const int32_t*>(uintptr_t(256)) : nullptr;
+    int rc = check_gate_args(aligned_stand_in, n_groups, N, stride, K, norm_mode, stop);
+    if (rc != SR_OK) return rc;
+    if (n_groups == 0) return SR_OK;
+    const HostArena h = host_arena(n_groups, N, stride, K);
+    if (arena == nullptr || arena_bytes < h.total || (reinterpret_cast<uintptr_t>(arena) & 255) != 0)
+        return SR_ERR_WORKSPACE;
+    unsigned char* d = static_cast<unsigned char*>(arena);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t P = pairs_of(N);
+    SR_CUDA_TRY(cudaMemcpyAsync(d + h.off_seqs, seqs, (size_t)n_groups * N * stride * 4,
+                                cudaMemcpyHostToDevice, s));
+    if (lens)
+        SR_CUDA_TRY(cudaMemcpyAsync(d + h.off_lens, lens, (size_t)n_groups * N * 4,
+                                    cudaMemcpyHostToDevice, s));
+    if (status)
+        SR_CUDA_TRY(cudaMemcpyAsync(d + h.off_status, status, 4, cudaMemcpyHostToDevice, s));
+    rc = sr_gate(reinterpret_cast<const int32_t*>(d + h.off_seqs),
+                 lens ? reinterpret_cast<const int32_t*>(d + h.off_lens) : nullptr, n_groups, N,
+                 stride, K, threshold, norm_mode,
+                 pair_dist ? reinterpret_cast<int32_t*>(d + h.off_dist) : nullptr,
+                 pair_sum ? reinterpret_cast<int32_t*>(d + h.off_sum) : nullptr,
+                 mean ? reinterpret_cast<double*>(d + h.off_mean) : nullptr, d + h.off_stop,
+                 status ? reinterpret_cast<int32_t*>(d + h.off_status) : nullptr, d + h.off_ws,
+                 h.total - h.off_ws, stream);
+    if (rc != SR_OK) return rc;
+    if (pair_dist)
+        SR_CUDA_TRY(cudaMemcpyAsync(pair_dist, d + h.off_dist, (size_t)n_groups * P * 4,
+                                    cudaMemcpyDeviceToHost, s));
+    if (pair_sum)
+        SR_CUDA_TRY(cudaMemcpyAsync(pair_sum, d + h.off_sum, (size_t)n_groups * 4,
+                                    cudaMemcpyDeviceToHost, s));
+    if (mean)
+        SR_CUDA_TRY(cudaMemcpyAsync(mean, d + h.off_mean, (size_t)n_groups * 8,
+                                    cudaMemcpyDeviceToHost, s));
+    SR_CUDA_TRY(cudaMemcpyAsync(stop, d + h.off_stop, (size_t)n_groups, cudaMemcpyDeviceToHost, s));
+    if (status)
+        SR_CUDA_TRY(cudaMemcpyAsync(status, d + h.off_status, 4, cudaMemcpyDeviceToHost, s));
+    return SR_OK;
+}
+
+size_t sr_incr_state_bytes(int32_t n_groups, int32_t N, int32_t max_steps) {
+    return incr_state_bytes(n_groups, N, max_steps);
+}
+
+int sr_incr_init(void* state, size_t state_bytes, int32_t n_groups, int32_t N, int32_t max_steps,
+                 void* stream) {
+    if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;
+    if (max_steps < 1 || max_steps > SR_MAX_INCR_STEPS) return SR_ERR_BAD_K;
+    if (state == nullptr) return SR_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(state) & 15) != 0) return SR_ERR_ALIGN;
+    return launch_incr_init(state, state_bytes, n_groups, N, max_steps,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int sr_gate_step_incremental(void* state, size_t state_bytes, const int32_t* new_actions,
+                             int32_t n_groups, int32_t N, double threshold, int32_t norm_mode,
+                             int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                             int32_t* status, void* stream) {
+    if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;
+    if (norm_mode != SR_NORM_MAXLEN && norm_mode != SR_NORM_NONE) return SR_ERR_BAD_MODE;
+    if (state == nullptr) return SR_ERR_NULL;
+    if (n_groups > 0 && (new_actions == nullptr || stop == nullptr)) return SR_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(state) & 15) != 0) return SR_ERR_ALIGN;
+    return launch_incr_step(state, state_bytes, new_actions, n_groups, N, threshold, norm_mode,
+                            pair_dist, pair_sum, mean, stop, status,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int sr_grpo_advantage(const float* rewards, const uint8_t* drop_mask, int32_t n_groups, int32_t N,
+                      float eps, float* adv, uint8_t* zero_var, void* stream) {
+    if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;
+    if (n_groups > 0 && (rewards == nullptr || adv == nullptr)) return SR_ERR_NULL;
+    return launch_advantage(rewards, drop_mask, n_groups, N, eps, adv, zero_var,
+                            static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

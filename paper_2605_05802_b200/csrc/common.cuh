@@ -1,0 +1,93 @@
+// Shared declarations of the sr_gate CUDA library (internal; the public boundary is include/sr_gate.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "sr_gate.h"
+
+namespace sr {
+
+// Records the text of a failed CUDA call for sr_last_cuda_error().
+void note_cuda_error(cudaError_t e, const char* where);
+
+#define SR_CUDA_TRY(expr)                                   \
+    do {                                                    \
+        cudaError_t e__ = (expr);                           \
+        if (e__ != cudaSuccess) {                           \
+            ::sr::note_cuda_error(e__, #expr);              \
+            return SR_ERR_CUDA;                             \
+        }                                                   \
+    } while (0)
+
+// Launch-error check that does not synchronise.
+#define SR_LAUNCH_CHECK(name)                               \
+    do {                                                    \
+        cudaError_t e__ = cudaGetLastError();               \
+        if (e__ != cudaSuccess) {                           \
+            ::sr::note_cuda_error(e__, name);               \
+            return SR_ERR_CUDA;                             \
+        }                                                   \
+    } while (0)
+
+struct GateArgs {
+    const int32_t* seqs;
+    const int32_t* lens;
+    int32_t n_groups, N, stride, K;
+    double threshold;
+    int32_t norm_mode;
+    int32_t* pair_dist;
+    int32_t* pair_sum;
+    double* mean;
+    uint8_t* stop;
+    int32_t* status;
+};
+
+__host__ __device__ inline int pairs_of(int N) { return N * (N - 1) / 2; }
+
+// Index of pair (a, b), a < b, in the order (0,1),(0,2),...,(N-2,N-1).
+__host__ __device__ inline int pair_index(int a, int b, int N) {
+    return a * N - a * (a + 1) / 2 + (b - a - 1);
+}
+
+// Inverse of pair_index.
+__device__ inline void pair_from_index(int p, int N, int& a, int& b) {
+    int i = 0, rem = p, row = N - 1;
+    while (rem >= row) { rem -= row; --row; ++i; }
+    a = i;
+    b = i + 1 + rem;
+}
+
+__device__ __forceinline__ uint32_t low_mask(int m) {   // m in 0..32
+    return m >= 32 ? 0xFFFFFFFFu : ((1u << m) - 1u);
+}
+
+// One term of the d_K sum (Section 3.2): the pair distance divided by the longer
+// prefix length, 0 for two empty prefixes; the raw distance in SR_NORM_NONE.
+__device__ __forceinline__ double pair_term(int d, int mi, int mj, int norm_mode) {
+    if (norm_mode == SR_NORM_NONE) return (double)d;
+    const int longer = mi > mj ? mi : mj;
+    return longer > 0 ? __ddiv_rn((double)d, (double)longer) : 0.0;
+}
+
+size_t align_up(size_t x, size_t a);
+
+// gate_single.cu: prefixes of at most 32 symbols, one 32-bit word per pair.
+int launch_gate_single(const GateArgs& a, cudaStream_t s);
+// gate_multi.cu: prefixes of up to SR_MAX_K symbols, blocked multi-word.
+size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
+int launch_gate_multi(const GateArgs& a, void* ws, size_t ws_bytes, cudaStream_t s);
+// incremental.cu
+size_t incr_state_bytes(int32_t n_groups, int32_t N, int32_t max_steps);
+int launch_incr_init(void* state, size_t bytes, int32_t n_groups, int32_t N, int32_t max_steps,
+                     cudaStream_t s);
+int launch_incr_step(void* state, size_t bytes, const int32_t* new_actions, int32_t n_groups,
+                     int32_t N, double threshold, int32_t norm_mode, int32_t* pair_dist,
+                     int32_t* pair_sum, double* mean, uint8_t* stop, int32_t* status,
+                     cudaStream_t s);
+// advantage.cu
+int launch_advantage(const float* rewards, const uint8_t* drop_mask, int32_t n_groups, int32_t N,
+                     float eps, float* adv, uint8_t* zero_var, cudaStream_t s);
+
+}  // namespace sr

@@ -1,0 +1,439 @@
+// Multi-word gate: prefixes of 33..SR_MAX_K symbols (token-level gate; same
+// d_K of Section 3.2 of the paper, applied to token IDs).
+//
+// The edit-distance matrix of a pair is cut into 32-row blocks of the pattern; a
+// block keeps its +1 / -1 vertical deltas in two 32-bit words and is advanced one
+// text column at a time by the bit-vector recurrence, with the horizontal delta
+// leaving a block entering the block below.  The work is organised as a pipeline
+// of five launches on the caller's stream, sharing a caller-provided workspace:
+//
+//   prep     one CTA per (group, pattern rollout): hashes the pattern's symbols
+//            in shared memory, then translates every text paired with it into a
+//            "loc" stream: for text column c the position of the column's symbol in
+//            the pattern (0xFFFF: absent; bit 15 set: several occurrences, walk
+//            the pattern's chain).  A block's match word is then just
+//            1 << (loc - first_row_of_block), no table lookup.  Also bins the pairs
+//            by (team shape, text length).
+//   scan     one CTA: prefix sums of the bins, warp-task table.
+//   scatter  orders the pairs: big shapes first, similar text lengths adjacent.
+//   dp       persistent warps pull tasks.  A task is a warp of 32/T teams; a team of
+//            T lanes owns one pair, lane l holding R consecutive blocks (32*R rows)
+//            in registers.  Lanes are skewed by one column (lane l works on column
+//            s - l at step s); the delta words of a lane's last block reach the next
+//            lane by one warp shuffle per step.  All pairs of a task share (T, R) and
+//            have similar lengths, so the warp's lanes stay busy.
+//   finish   one thread per group: ordered fp64 sum of the normalised terms,
+//            threshold, outputs.
+//
+// Which rollout of a pair is the pattern is fixed by a round-robin tournament on the
+// indices, so that every pattern CTA of `prep` serves the same number of texts.
+#include "common.cuh"
+
+namespace sr {
+namespace {
+
+constexpr int kPrepThreads = 256;
+constexpr int kNumClasses = 16;     // class = log2(T) * 4 + (R - 1)
+constexpr int kLenBuckets = 64;     // text length / 16
+constexpr int kNumBins = kNumClasses * kLenBuckets;
+constexpr uint32_t kLocNone = 0xFFFFu;
+constexpr uint32_t kLocMulti = 0x8000u;
+constexpr uint32_t kChainEnd = 0xFFFFu;
+constexpr int kDpWarpsPerCta = 4;
+
+struct PairDesc {          // 16 bytes
+    uint32_t mn;           // m | n << 16
+    uint32_t pat_row;      // g * N + pattern rollout
+    uint32_t bin;          // bin index; bit 31 = pair needs the dp kernel
+    uint32_t pad;
+};
+
+struct Ctl {               // int32 control block in the workspace
+    int32_t hist[kNumBins];
+    int32_t start[kNumBins];
+    int32_t fill[kNumBins];
+    int32_t cls_pair_start[kNumClasses + 1];   // by descending class
+    int32_t cls_task_start[kNumClasses + 1];
+    int32_t task_counter;
+    int32_t total_tasks;
+};
+
+struct MultiWs {
+    size_t off_dist, off_desc, off_loc, off_next, off_order, off_ctl, total;
+    int pitch;             // uint16 elements per loc / chain row
+};
+
+MultiWs multi_layout(int32_t n_groups, int32_t N, int32_t K) {
+    MultiWs w;
+    const size_t P = pairs_of(N);
+    w.pitch = (K + 7) & ~7;
+    size_t off = 0;
+    w.off_ctl = off;   off = align_up(off + sizeof(Ctl), 256);
+    w.off_dist = off;  off = align_up(off + (size_t)n_groups * P * 4, 256);
+    w.off_desc = off;  off = align_up(off + (size_t)n_groups * P * sizeof(PairDesc), 256);
+    w.off_order = off; off = align_up(off + (size_t)n_groups * P * 4, 256);
+    w.off_next = off;  off = align_up(off + (size_t)n_groups * N * w.pitch * 2, 256);
+    w.off_loc = off;   off = align_up(off + (size_t)n_groups * P * w.pitch * 2, 256);
+    w.total = off;
+    return w;
+}
+
+// Pattern side of pair (a, b), a < b: a round-robin tournament in which every vertex
+// of an odd cycle beats the following half; with N even the last rollout is a text
+// for everyone.  Every pattern gets floor(N/2) texts (N even: N/2 for all but the last).
+__host__ __device__ inline bool first_is_pattern(int a, int b, int N) {
+    const int M = (N & 1) ? N : N - 1;
+    if (b >= M) return true;
+    return (b - a) <= (M - 1) / 2;
+}
+
+__host__ __device__ inline void team_shape(int m, int& tlog, int& R) {
+    const int W = (m + 31) >> 5;
+    if (W <= 4) { tlog = 0; R = W; }
+    else if (W <= 8) { tlog = 1; R = (W + 1) >> 1; }
+    else if (W <= 16) { tlog = 2; R = (W + 3) >> 2; }
+    else { tlog = 3; R = (W + 7) >> 3; }
+}
+
+__device__ __forceinline__ int clamp_len(const int32_t* lens, size_t idx, int K, bool& neg) {
+    int len = lens ? lens[idx] : K;
+    if (len < 0) { len = 0; neg = true; }
+    return min(len, K);
+}
+
+// ------------------------------------------------------------------------ prep
+__global__ void __launch_bounds__(kPrepThreads)
+multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots, int hshift,
+                  int32_t* dist_out) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    int32_t* s_pat = reinterpret_cast<int32_t*>(smem);                       // [pitch]
+    uint32_t* s_owner = reinterpret_cast<uint32_t*>(s_pat + W.pitch);        // [hslots]
+    uint32_t* s_head = s_owner + hslots;                                     // [hslots]
+    uint16_t* s_next = reinterpret_cast<uint16_t*>(s_head + hslots);         // [pitch]
+
+    const int N = a.N, K = a.K, P = pairs_of(N);
+    const int g = blockIdx.x / N, i = blockIdx.x - g * N;
+    const int tid = threadIdx.x;
+    const int M = (N & 1) ? N : N - 1;
+    if (i >= M) return;                               // the last rollout of an even group is never a pattern
+    bool neg = false;
+    const int m = clamp_len(a.lens, (size_t)g * N + i, K, neg);
+    const int32_t* pat = a.seqs + ((size_t)g * N + i) * a.stride;
+    for (int p = tid; p < m; p += kPrepThreads) s_pat[p] = __ldg(pat + p);
+    for (int h = tid; h < hslots; h += kPrepThreads) { s_owner[h] = 0u; s_head[h] = 0u; }
+    __syncthreads();
+    // every position claims (or finds) the slot of its symbol and pushes itself on
+    // the slot's occurrence chain
+    for (int p = tid; p < m; p += kPrepThreads) {
+        const int32_t sym = s_pat[p];
+        uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> hshift;
+        // at least twice as many slots as symbols: a free or matching slot always
+        // exists; the trip count is bounded all the same
+        for (int probe = 0; probe < hslots; ++probe) {
+            uint32_t o = s_owner[h];
+            if (o == 0u) o = atomicCAS(&s_owner[h], 0u, (uint32_t)p + 1u);
+            if (o == 0u || s_pat[o - 1u] == sym) break;
+            h = (h + 1u) & (uint32_t)(hslots - 1);
+        }
+        const uint32_t prev = atomicExch(&s_head[h], (uint32_t)p + 1u);
+        s_next[p] = prev == 0u ? (uint16_t)kChainEnd : (uint16_t)(prev - 1u);
+    }
+    __syncthreads();
+    uint16_t* g_next = reinterpret_cast<uint16_t*>(ws + W.off_next) + ((size_t)g * N + i) * W.pitch;
+    for (int p = tid; p < m; p += kPrepThreads) g_next[p] = s_next[p];
+
+    PairDesc* descs = reinterpret_cast<PairDesc*>(ws + W.off_desc);
+    uint16_t* locs = reinterpret_cast<uint16_t*>(ws + W.off_loc);
+    Ctl* ctl = reinterpret_cast<Ctl*>(ws + W.off_ctl);
+    int tlog, R;
+    team_shape(m, tlog, R);
+    const int cls = tlog * 4 + (R - 1);
+    for (int j = 0; j < N; ++j) {
+        if (j == i) continue;
+        const int lo = min(i, j), hi = max(i, j);
+        if (first_is_pattern(lo, hi, N) != (lo == i)) continue;
+        const int n = clamp_len(a.lens, (size_t)g * N + j, K, neg);
+        const size_t idx = (size_t)g * P + pair_index(lo, hi, N);
+        if (m == 0 || n == 0) {
+            if (tid == 0) {
+                dist_out[idx] = max(m, n);
+                descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i), 0u, 0u};
+            }
+            continue;
+        }
+        const int32_t* txt = a.seqs + ((size_t)g * N + j) * a.stride;
+        uint16_t* loc = locs + idx * W.pitch;
+        for (int c = tid; c < n; c += kPrepThreads) {
+            const int32_t sym = __ldg(txt + c);
+            uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> hshift;
+            uint32_t v = kLocNone;
+            for (int probe = 0; probe < hslots; ++probe) {
+                const uint32_t o = s_owner[h];
+                if (o == 0u) break;
+                if (s_pat[o - 1u] == sym) {
+                    const uint32_t first = s_head[h] - 1u;
+                    v = s_next[first] == kChainEnd ? first : (kLocMulti | first);
+                    break;
+                }
+                h = (h + 1u) & (uint32_t)(hslots - 1);
+            }
+            loc[c] = (uint16_t)v;
+        }
+        if (tid == 0) {
+            const int bucket = min(n >> 4, kLenBuckets - 1);
+            const int bin = (kNumClasses - 1 - cls) * kLenBuckets + (kLenBuckets - 1 - bucket);
+            descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i),
+                                  (uint32_t)bin | 0x80000000u, 0u};
+            atomicAdd(&ctl->hist[bin], 1);
+        }
+    }
+    if (neg && tid == 0 && a.status) atomicOr(a.status, SR_STATUS_NEG_LEN);
+}
+
+// ------------------------------------------------------------------------ scan
+__global__ void __launch_bounds__(kNumBins)
+multi_scan_kernel(Ctl* ctl) {
+    __shared__ int32_t s[kNumBins];
+    const int t = threadIdx.x;
+    const int own = ctl->hist[t];
+    s[t] = own;
+    __syncthreads();
+    for (int d = 1; d < kNumBins; d <<= 1) {
+        const int v = t >= d ? s[t - d] : 0;
+        __syncthreads();
+        s[t] += v;
+        __syncthreads();
+    }
+    ctl->start[t] = s[t] - own;
+    ctl->fill[t] = 0;
+    ctl->hist[t] = 0;                  // ready for the next call on this workspace
+    if (t == 0) {
+        int tasks = 0;
+        for (int k = 0; k < kNumClasses; ++k) {          // k-th class by descending size
+            const int cls = kNumClasses - 1 - k;
+            const int first = k * kLenBuckets;
+            const int begin = first == 0 ? 0 : s[first - 1];
+            const int end = s[first + kLenBuckets - 1];
+            const int tpw = 32 >> (cls >> 2);
+            ctl->cls_pair_start[k] = begin;
+            ctl->cls_task_start[k] = tasks;
+            tasks += (end - begin + tpw - 1) / tpw;
+            if (k == kNumClasses - 1) {
+                ctl->cls_pair_start[kNumClasses] = end;
+                ctl->cls_task_start[kNumClasses] = tasks;
+            }
+        }
+        ctl->total_tasks = tasks;
+        ctl->task_counter = 0;
+    }
+}
+
+// --------------------------------------------------------------------- scatter
+__global__ void __launch_bounds__(256)
+multi_scatter_kernel(const PairDesc* descs, int32_t* order, Ctl* ctl, int n_pairs) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n_pairs) return;
+    const uint32_t b = descs[idx].bin;
+    if (!(b & 0x80000000u)) return;
+    const int bin = (int)(b & 0x7FFFFFFFu);
+    const int pos = ctl->start[bin] + atomicAdd(&ctl->fill[bin], 1);
+    order[pos] = idx;
+}
+
+// -------------------------------------------------------------------------- dp
+__device__ __forceinline__ uint32_t shl_clamp(uint32_t v, uint32_t s) {
+    uint32_t r;   // PTX shl clamps shift amounts above 31: the result is 0
+    asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(s));
+    return r;
+}
+
+template <int R>
+__device__ __forceinline__ void dp_task(int tlog, int pos, bool valid, const PairDesc* descs,
+                                        const int32_t* order, const uint16_t* locs,
+                                        const uint16_t* nexts, int pitch, int32_t* dist_out) {
+    const int lane = threadIdx.x & 31;
+    const int T = 1 << tlog;
+    const int lt = lane & (T - 1);
+    int idx = 0, m = 0, n = 0;
+    const uint16_t* loc = locs;
+    const uint16_t* nxt = nexts;
+    if (valid) {
+        idx = order[pos];
+        const PairDesc d = descs[idx];
+        m = (int)(d.mn & 0xFFFFu);
+        n = (int)(d.mn >> 16);
+        loc = locs + (size_t)idx * pitch;
+        nxt = nexts + (size_t)d.pat_row * pitch;
+    }
+    const int rowbase = lt * R * 32;
+    int nsteps = valid ? n + T - 1 : 0;
+    nsteps = __reduce_max_sync(0xFFFFFFFFu, nsteps);
+
+    uint32_t Pv[R], Mv[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) { Pv[r] = 0xFFFFFFFFu; Mv[r] = 0u; }
+    uint32_t lastP = 0u, lastM = 0u;
+    uint32_t loc_nxt = (valid && lt == 0) ? (uint32_t)__ldg(loc) : kLocNone;
+
+    for (int s = 0; s < nsteps; ++s) {
+        const int c = s - lt;
+        const bool active = valid && c >= 0 && c < n;
+        const uint32_t loc_now = loc_nxt;
+        {
+            const int cn = c + 1;
+            loc_nxt = (valid && cn >= 0 && cn < n) ? (uint32_t)__ldg(loc + cn) : kLocNone;
+        }
+        // horizontal deltas leaving the lane above (its previous step = this column)
+        uint32_t inP = __shfl_up_sync(0xFFFFFFFFu, lastP, 1);
+        uint32_t inM = __shfl_up_sync(0xFFFFFFFFu, lastM, 1);
+        if (lt == 0) { inP = 0x80000000u; inM = 0u; }      // row 0: D[0][c] - D[0][c-1] = +1
+        if (active) {
+            const uint32_t d0 = loc_now - (uint32_t)rowbase;
+            uint32_t Eq[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) Eq[r] = shl_clamp(1u, d0 - 32u * r);
+            if (loc_now >= kLocMulti && loc_now != kLocNone) {
+                uint32_t p = loc_now & 0x7FFFu;
+                for (int hop = 0; hop < SR_MAX_K && p < (uint32_t)m; ++hop) {   // chain ends at 0xFFFF
+                    const uint32_t dd = p - (uint32_t)rowbase;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) Eq[r] |= shl_clamp(1u, dd - 32u * r);
+                    p = __ldg(nxt + p);
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const uint32_t pv = Pv[r], mv = Mv[r];
+                const uint32_t Xv = Eq[r] | mv;
+                const uint32_t Eh = Eq[r] | (inM >> 31);
+                const uint32_t Xh = (((Eh & pv) + pv) ^ pv) | Eh;
+                const uint32_t Ph = mv | ~(Xh | pv);
+                const uint32_t Mh = pv & Xh;
+                const uint32_t Phs = __funnelshift_l(inP, Ph, 1);
+                const uint32_t Mhs = __funnelshift_l(inM, Mh, 1);
+                Pv[r] = Mhs | ~(Xv | Phs);
+                Mv[r] = Phs & Xv;
+                inP = Ph;
+                inM = Mh;
+            }
+            lastP = inP;
+            lastM = inM;
+        }
+    }
+    // D[m][n] = n + (sum of the vertical deltas of the last column over rows 1..m)
+    int part = 0;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int rows = min(max(m - (rowbase + 32 * r), 0), 32);
+        const uint32_t msk = low_mask(rows);
+        part += __popc(Pv[r] & msk) - __popc(Mv[r] & msk);
+    }
+    for (int off = 1; off < T; off <<= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, off);
+    if (valid && lt == 0) dist_out[idx] = n + part;
+}
+
+__global__ void __launch_bounds__(kDpWarpsPerCta * 32)
+multi_dp_kernel(unsigned char* ws, MultiWs W, int32_t* dist_out) {
+    Ctl* ctl = reinterpret_cast<Ctl*>(ws + W.off_ctl);
+    const PairDesc* descs = reinterpret_cast<const PairDesc*>(ws + W.off_desc);
+    const int32_t* order = reinterpret_cast<const int32_t*>(ws + W.off_order);
+    const uint16_t* locs = reinterpret_cast<const uint16_t*>(ws + W.off_loc);
+    const uint16_t* nexts = reinterpret_cast<const uint16_t*>(ws + W.off_next);
+    const int lane = threadIdx.x & 31;
+    const int total = ctl->total_tasks;
+    while (true) {
+        int task = 0;
+        if (lane == 0) task = atomicAdd(&ctl->task_counter, 1);
+        task = __shfl_sync(0xFFFFFFFFu, task, 0);
+        if (task >= total) break;
+        int k = 0;
+        while (k + 1 < kNumClasses && task >= ctl->cls_task_start[k + 1]) ++k;
+        const int cls = kNumClasses - 1 - k;
+        const int tlog = cls >> 2, R = (cls & 3) + 1;
+        const int tpw = 32 >> tlog;
+        const int pos = ctl->cls_pair_start[k] + (task - ctl->cls_task_start[k]) * tpw + (lane >> tlog);
+        const bool valid = pos < ctl->cls_pair_start[k + 1];
+        switch (R) {
+            case 1: dp_task<1>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out); break;
+            case 2: dp_task<2>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out); break;
+            case 3: dp_task<3>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out); break;
+            default: dp_task<4>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out); break;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------- finish
+__global__ void __launch_bounds__(128)
+multi_finish_kernel(GateArgs a, const int32_t* dist) {
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= a.n_groups) return;
+    const int N = a.N, P = pairs_of(N);
+    bool neg = false;
+    double s = 0.0;
+    int isum = 0, p = 0;
+    for (int i = 0; i < N; ++i) {
+        const int mi = clamp_len(a.lens, (size_t)g * N + i, a.K, neg);
+        for (int j = i + 1; j < N; ++j, ++p) {
+            const int mj = clamp_len(a.lens, (size_t)g * N + j, a.K, neg);
+            const int d = dist[(size_t)g * P + p];
+            isum += d;
+            s = __dadd_rn(s, pair_term(d, mi, mj, a.norm_mode));
+        }
+    }
+    const double dk = __ddiv_rn(s, (double)P);
+    if (a.pair_sum) a.pair_sum[g] = isum;
+    if (a.mean) a.mean[g] = dk;
+    a.stop[g] = dk < a.threshold ? 1 : 0;
+}
+
+}  // namespace
+
+size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K) {
+    (void)stride;
+    return multi_layout(n_groups, N, K).total;
+}
+
+int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_t s) {
+    if (a.n_groups == 0) return SR_OK;
+    const MultiWs W = multi_layout(a.n_groups, a.N, a.K);
+    if (ws_ == nullptr || ws_bytes < W.total || (reinterpret_cast<uintptr_t>(ws_) & 255) != 0)
+        return SR_ERR_WORKSPACE;
+    unsigned char* ws = static_cast<unsigned char*>(ws_);
+    const int P = pairs_of(a.N);
+    const long long n_pairs_ll = (long long)a.n_groups * P;
+    if (n_pairs_ll > 0x7FFFFFFFLL) return SR_ERR_BAD_N;
+    const int n_pairs = (int)n_pairs_ll;
+    int32_t* dist = a.pair_dist ? a.pair_dist : reinterpret_cast<int32_t*>(ws + W.off_dist);
+    Ctl* ctl = reinterpret_cast<Ctl*>(ws + W.off_ctl);
+
+    int hslots = 64;
+    while (hslots < 2 * a.K) hslots <<= 1;
+    int hshift = 32;
+    while ((1 << (32 - hshift)) < hslots) --hshift;
+    const int prep_smem = W.pitch * 4 + hslots * 8 + W.pitch * 2;
+
+    SR_CUDA_TRY(cudaMemsetAsync(ctl->hist, 0, sizeof(ctl->hist), s));
+    multi_prep_kernel<<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, hshift, dist);
+    SR_LAUNCH_CHECK("multi_prep_kernel");
+    multi_scan_kernel<<<1, kNumBins, 0, s>>>(ctl);
+    SR_LAUNCH_CHECK("multi_scan_kernel");
+    multi_scatter_kernel<<<(n_pairs + 255) / 256, 256, 0, s>>>(
+        reinterpret_cast<const PairDesc*>(ws + W.off_desc),
+        reinterpret_cast<int32_t*>(ws + W.off_order), ctl, n_pairs);
+    SR_LAUNCH_CHECK("multi_scatter_kernel");
+    int dev = 0, sms = 0;
+    SR_CUDA_TRY(cudaGetDevice(&dev));
+    SR_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    // persistent grid: a multiple of the SM count; warps pull tasks until none is left
+    long long want = (n_pairs_ll + kDpWarpsPerCta - 1) / kDpWarpsPerCta;
+    long long cap = (long long)sms * 12;
+    int blocks = (int)(want < cap ? want : cap);
+    if (blocks < 1) blocks = 1;
+    multi_dp_kernel<<<blocks, kDpWarpsPerCta * 32, 0, s>>>(ws, W, dist);
+    SR_LAUNCH_CHECK("multi_dp_kernel");
+    multi_finish_kernel<<<(a.n_groups + 127) / 128, 128, 0, s>>>(a, dist);
+    SR_LAUNCH_CHECK("multi_finish_kernel");
+    return SR_OK;
+}
+
+}  // namespace sr

@@ -1,0 +1,282 @@
+// Incremental gate: one new action per rollout per environment step, gate
+// re-evaluated after every step (the paper gates at one fixed K, Appendix C.1; a
+// per-step evaluation is what its "adaptive K" follow-up needs, Section 5).
+//
+// Per pair (i, j), i < j, with current lengths m = len_i (rows) and n = len_j
+// (columns) of the edit-distance matrix D, the state keeps
+//   VP / VN : bit r-1 set iff D[r][n] - D[r-1][n] is +1 / -1   (last column)
+//   HP / HN : bit c-1 set iff D[m][c] - D[m][c-1] is +1 / -1   (last row)
+// and D[m][n] = n + popc(VP) - popc(VN) is never stored.  When j appends y, one
+// bit-parallel column step over the rows gives the new last column and the
+// horizontal delta of the bottom row; when i appends x, the same step on the
+// transposed roles gives the new last row; when both append, both steps start from
+// the OLD state and the new corner D[m+1][n+1] is the usual three-way minimum.
+//
+// State buffer layout (position independent, byte-copyable):
+//   [0, 256)        header: magic, n_groups, N, max_steps
+//   lens   int32 [n_groups][N]
+//   hist   int32 [n_groups][N][32]        actions emitted so far
+//   pairs  uint4 [n_groups][P]            (VP, VN, HP, HN)
+// every section starts on a 256-byte boundary.
+#include "common.cuh"
+
+namespace sr {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+namespace {
+
+constexpr uint32_t kMagic = 0x53524731u;   // "SRG1"
+constexpr int kHistPitch = 32;
+
+struct IncrLayout {
+    size_t off_lens, off_hist, off_pairs, total;
+};
+
+IncrLayout incr_layout(int32_t n_groups, int32_t N) {
+    IncrLayout L;
+    size_t off = 256;
+    L.off_lens = off;
+    off = align_up(off + (size_t)n_groups * N * 4, 256);
+    L.off_hist = off;
+    off = align_up(off + (size_t)n_groups * N * kHistPitch * 4, 256);
+    L.off_pairs = off;
+    off = align_up(off + (size_t)n_groups * pairs_of(N) * 16, 256);
+    L.total = off;
+    return L;
+}
+
+__global__ void incr_init_kernel(unsigned char* state, IncrLayout L, int n_groups, int N,
+                                 int max_steps) {
+    const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t nthr = (size_t)gridDim.x * blockDim.x;
+    uint32_t* hdr = reinterpret_cast<uint32_t*>(state);
+    if (tid < 64) {
+        uint32_t v = 0;
+        if (tid == 0) v = kMagic;
+        if (tid == 1) v = (uint32_t)n_groups;
+        if (tid == 2) v = (uint32_t)N;
+        if (tid == 3) v = (uint32_t)max_steps;
+        hdr[tid] = v;
+    }
+    // lengths and pair state start at zero; the history needs no clearing (only the
+    // first len entries of a row are ever read)
+    uint32_t* lens = reinterpret_cast<uint32_t*>(state + L.off_lens);
+    for (size_t e = tid; e < (size_t)n_groups * N; e += nthr) lens[e] = 0u;
+    uint4* pairs = reinterpret_cast<uint4*>(state + L.off_pairs);
+    for (size_t e = tid; e < (size_t)n_groups * pairs_of(N); e += nthr)
+        pairs[e] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// One bit-parallel column step over `m` rows (m >= 1) with horizontal input +1 at
+// row 0; returns the horizontal delta leaving the bottom row.
+__device__ __forceinline__ int column_step(uint32_t Eq, uint32_t& Pv, uint32_t& Mv, int m) {
+    const uint32_t Xv = Eq | Mv;
+    const uint32_t Xh = (((Eq & Pv) + Pv) ^ Pv) | Eq;
+    uint32_t Ph = Mv | ~(Xh | Pv);
+    uint32_t Mh = Pv & Xh;
+    const int hout = (int)((Ph >> (m - 1)) & 1u) - (int)((Mh >> (m - 1)) & 1u);
+    Ph = (Ph << 1) | 1u;
+    Mh = Mh << 1;
+    const uint32_t msk = low_mask(m);
+    Pv = (Mh | ~(Xv | Ph)) & msk;
+    Mv = (Ph & Xv) & msk;
+    return hout;
+}
+
+struct IncrArgs {
+    unsigned char* state;
+    IncrLayout L;
+    const int32_t* new_actions;
+    int n_groups, N;
+    double threshold;
+    int norm_mode;
+    int32_t* pair_dist;
+    int32_t* pair_sum;
+    double* mean;
+    uint8_t* stop;
+    int32_t* status;
+    int gpb;
+    int off_len, off_new, off_hist, off_dist, off_term, off_pairs;   // shared-memory offsets
+};
+
+__global__ void __launch_bounds__(1024)
+incr_step_kernel(IncrArgs a) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int N = a.N, P = pairs_of(N);
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int g0 = blockIdx.x * a.gpb;
+    const int ng = min(a.gpb, a.n_groups - g0);
+    const uint32_t* hdr = reinterpret_cast<const uint32_t*>(a.state);
+    if (hdr[0] != kMagic || hdr[1] != (uint32_t)a.n_groups || hdr[2] != (uint32_t)N) {
+        if (tid == 0 && a.status) atomicOr(a.status, SR_STATUS_BAD_STATE);
+        return;
+    }
+    const int max_steps = (int)hdr[3];
+
+    int32_t* s_len = reinterpret_cast<int32_t*>(smem + a.off_len);      // [gpb][N] old lengths
+    int32_t* s_new = reinterpret_cast<int32_t*>(smem + a.off_new);      // [gpb][N] new action
+    int32_t* s_hist = reinterpret_cast<int32_t*>(smem + a.off_hist);    // [gpb][N][33]
+    int32_t* s_dist = reinterpret_cast<int32_t*>(smem + a.off_dist);    // [gpb][P]
+    double* s_term = reinterpret_cast<double*>(smem + a.off_term);      // [gpb][P]
+    uint16_t* s_pairs = reinterpret_cast<uint16_t*>(smem + a.off_pairs);
+
+    int32_t* g_len = reinterpret_cast<int32_t*>(a.state + a.L.off_lens) + (size_t)g0 * N;
+    int32_t* g_hist = reinterpret_cast<int32_t*>(a.state + a.L.off_hist) + (size_t)g0 * N * kHistPitch;
+    uint4* g_pairs = reinterpret_cast<uint4*>(a.state + a.L.off_pairs) + (size_t)g0 * P;
+
+    bool overflow = false;
+    for (int e = tid; e < ng * N; e += nthr) {
+        const int len = g_len[e];
+        int32_t act = __ldg(a.new_actions + (size_t)g0 * N + e);
+        if (act != SR_NO_ACTION && len >= max_steps) { act = SR_NO_ACTION; overflow = true; }
+        s_len[e] = len;
+        s_new[e] = act;
+    }
+    if (overflow && a.status) atomicOr(a.status, SR_STATUS_STEP_OVERFLOW);
+    for (int p = tid; p < P; p += nthr) {
+        int i, j;
+        pair_from_index(p, N, i, j);
+        s_pairs[p] = (uint16_t)(i | (j << 8));
+    }
+    __syncthreads();
+    // history so far -> shared memory (rows padded to 33 words: pair threads of one
+    // warp read different rows at the same position)
+    for (int e = tid; e < ng * N * kHistPitch; e += nthr) {
+        const int row = e >> 5, r = e & 31;
+        if (r < s_len[row]) s_hist[row * 33 + r] = g_hist[e];
+    }
+    __syncthreads();
+    // append this step's actions to the stored history and lengths
+    for (int e = tid; e < ng * N; e += nthr) {
+        if (s_new[e] != SR_NO_ACTION) {
+            g_hist[e * kHistPitch + s_len[e]] = s_new[e];
+            g_len[e] = s_len[e] + 1;
+        }
+    }
+
+    if (tid < ng * P) {
+        const int g = tid / P, p = tid - g * P;
+        const int pr = s_pairs[p];
+        const int i = pr & 0xFF, j = pr >> 8;
+        const int m = s_len[g * N + i], n = s_len[g * N + j];
+        const int32_t x = s_new[g * N + i], y = s_new[g * N + j];
+        const bool ai = x != SR_NO_ACTION, aj = y != SR_NO_ACTION;
+        uint4 st = g_pairs[tid];
+        uint32_t VP = st.x, VN = st.y, HP = st.z, HN = st.w;
+        const int c = n + __popc(VP) - __popc(VN);
+        int hout = 1, vout = 1;
+        uint32_t VP2 = VP, VN2 = VN, HP2 = HP, HN2 = HN;
+        if (aj && m > 0) {
+            const int32_t* hi = s_hist + (g * N + i) * 33;
+            uint32_t Eq = 0u;
+            for (int r = 0; r < m; ++r) Eq |= (hi[r] == y ? 1u : 0u) << r;
+            hout = column_step(Eq, VP2, VN2, m);
+        }
+        if (ai && n > 0) {
+            const int32_t* hj = s_hist + (g * N + j) * 33;
+            uint32_t Eq = 0u;
+            for (int r = 0; r < n; ++r) Eq |= (hj[r] == x ? 1u : 0u) << r;
+            vout = column_step(Eq, HP2, HN2, n);
+        }
+        int d = c, mi = m, mj = n;
+        if (ai && aj) {
+            const int left = c + vout, up = c + hout;
+            d = min(min(c + (x != y ? 1 : 0), up + 1), left + 1);
+            const int vd = d - up, hd = d - left;
+            VP = VP2 | (vd > 0 ? 1u << m : 0u);
+            VN = VN2 | (vd < 0 ? 1u << m : 0u);
+            HP = HP2 | (hd > 0 ? 1u << n : 0u);
+            HN = HN2 | (hd < 0 ? 1u << n : 0u);
+            mi = m + 1; mj = n + 1;
+        } else if (aj) {
+            d = c + hout;
+            VP = VP2; VN = VN2;
+            HP |= hout > 0 ? 1u << n : 0u;
+            HN |= hout < 0 ? 1u << n : 0u;
+            mj = n + 1;
+        } else if (ai) {
+            d = c + vout;
+            HP = HP2; HN = HN2;
+            VP |= vout > 0 ? 1u << m : 0u;
+            VN |= vout < 0 ? 1u << m : 0u;
+            mi = m + 1;
+        }
+        if (ai || aj) g_pairs[tid] = make_uint4(VP, VN, HP, HN);
+        s_dist[tid] = d;
+        s_term[tid] = pair_term(d, mi, mj, a.norm_mode);
+        if (a.pair_dist) a.pair_dist[(size_t)g0 * P + tid] = d;
+    }
+    __syncthreads();
+    if (tid < ng) {
+        double s = 0.0;
+        int isum = 0;
+        for (int p = 0; p < P; ++p) {
+            s = __dadd_rn(s, s_term[tid * P + p]);
+            isum += s_dist[tid * P + p];
+        }
+        const double dk = __ddiv_rn(s, (double)P);
+        if (a.pair_sum) a.pair_sum[g0 + tid] = isum;
+        if (a.mean) a.mean[g0 + tid] = dk;
+        a.stop[g0 + tid] = dk < a.threshold ? 1 : 0;
+    }
+}
+
+}  // namespace
+
+size_t incr_state_bytes(int32_t n_groups, int32_t N, int32_t max_steps) {
+    if (n_groups < 0 || N < 2 || N > SR_MAX_N || max_steps < 1 || max_steps > SR_MAX_INCR_STEPS)
+        return 0;
+    return incr_layout(n_groups, N).total;
+}
+
+int launch_incr_init(void* state, size_t bytes, int32_t n_groups, int32_t N, int32_t max_steps,
+                     cudaStream_t s) {
+    const IncrLayout L = incr_layout(n_groups, N);
+    if (bytes < L.total) return SR_ERR_STATE_SIZE;
+    size_t work = (size_t)n_groups * pairs_of(N);
+    int blocks = (int)((work + 255) / 256);
+    if (blocks < 1) blocks = 1;
+    if (blocks > 4096) blocks = 4096;
+    incr_init_kernel<<<blocks, 256, 0, s>>>(static_cast<unsigned char*>(state), L, n_groups, N, max_steps);
+    SR_LAUNCH_CHECK("incr_init_kernel");
+    return SR_OK;
+}
+
+int launch_incr_step(void* state, size_t bytes, const int32_t* new_actions, int32_t n_groups,
+                     int32_t N, double threshold, int32_t norm_mode, int32_t* pair_dist,
+                     int32_t* pair_sum, double* mean, uint8_t* stop, int32_t* status,
+                     cudaStream_t s) {
+    IncrArgs a;
+    a.L = incr_layout(n_groups, N);
+    if (bytes < a.L.total) return SR_ERR_STATE_SIZE;
+    if (n_groups == 0) return SR_OK;
+    a.state = static_cast<unsigned char*>(state);
+    a.new_actions = new_actions;
+    a.n_groups = n_groups; a.N = N;
+    a.threshold = threshold; a.norm_mode = norm_mode;
+    a.pair_dist = pair_dist; a.pair_sum = pair_sum; a.mean = mean; a.stop = stop; a.status = status;
+    const int P = pairs_of(N);
+    int gpb = 256 / P;
+    if (gpb < 1) gpb = 1;
+    if (gpb > 32) gpb = 32;
+    a.gpb = gpb;
+    int off = 0;
+    auto take = [&](int b) { int o = off; off = (off + b + 15) & ~15; return o; };
+    a.off_len = take(gpb * N * 4);
+    a.off_new = take(gpb * N * 4);
+    a.off_hist = take(gpb * N * 33 * 4);
+    a.off_dist = take(gpb * P * 4);
+    a.off_term = take(gpb * P * 8);
+    a.off_pairs = take(P * 2);
+    int threads = (gpb * P + 31) & ~31;
+    if (threads < 64) threads = 64;
+    if (off > 48 * 1024)
+        SR_CUDA_TRY(cudaFuncSetAttribute(incr_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, off));
+    const int blocks = (n_groups + gpb - 1) / gpb;
+    incr_step_kernel<<<blocks, threads, off, s>>>(a);
+    SR_LAUNCH_CHECK("incr_step_kernel");
+    return SR_OK;
+}
+
+}  // namespace sr

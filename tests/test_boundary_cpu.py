@@ -1,0 +1,120 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every
+symbol the headers declare, and rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2605_05802_b200 as sr
+from paper_2605_05802_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load()
+
+
+def _declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in sorted(os.listdir(inc)):
+        text = open(os.path.join(inc, f)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(sr_[a-z0-9_]+)\s*\(", text))
+    return names
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert {"sr_gate", "sr_gate_step_incremental", "sr_grpo_advantage", "sr_incr_init",
+            "sr_gate_host", "sr_probe_int32"} <= names
+    for n in names:
+        assert hasattr(lib, n), n
+    assert names == set(binding._SIGNATURES), names ^ set(binding._SIGNATURES)
+    assert lib.sr_version() == 100
+
+
+def test_strerror_is_total(lib):
+    for code in range(-9, 1):
+        assert lib.sr_strerror(code)
+    assert b"unknown" in lib.sr_strerror(-99)
+
+
+def test_gate_rejects_bad_arguments_before_any_launch(lib):
+    fake = 1 << 20          # never dereferenced: every call below fails validation
+    def gate(seqs=fake, lens=None, G=4, N=8, stride=32, K=10, thr=0.12, mode=0, stop=fake,
+             ws=None, wsb=0):
+        return lib.sr_gate(seqs, lens, G, N, stride, K, thr, mode, None, None, None, stop, None,
+                           ws, wsb, None)
+    assert gate(N=1) == binding.SR_ERR_BAD_N
+    assert gate(N=33) == binding.SR_ERR_BAD_N
+    assert gate(G=-1) == binding.SR_ERR_BAD_N
+    assert gate(K=-1) == binding.SR_ERR_BAD_K
+    assert gate(K=33) == binding.SR_ERR_BAD_K            # K > stride
+    assert gate(stride=2048, K=1025) == binding.SR_ERR_BAD_K
+    assert gate(mode=2) == binding.SR_ERR_BAD_MODE
+    assert gate(seqs=None) == binding.SR_ERR_NULL
+    assert gate(stop=None) == binding.SR_ERR_NULL
+    assert gate(stride=30, K=10) == binding.SR_ERR_ALIGN
+    assert gate(seqs=fake + 4) == binding.SR_ERR_ALIGN
+    # multi-word path needs a workspace
+    assert gate(stride=64, K=64) == binding.SR_ERR_WORKSPACE
+    assert gate(stride=64, K=64, ws=fake, wsb=16) == binding.SR_ERR_WORKSPACE
+    assert gate(stride=64, K=64, ws=fake + 8, wsb=1 << 30) == binding.SR_ERR_WORKSPACE
+    # an empty batch is a valid no-op on either path
+    assert gate(G=0, seqs=None, stop=None) == binding.SR_OK
+    assert gate(G=0, seqs=None, stop=None, stride=64, K=64) == binding.SR_OK
+
+
+def test_workspace_and_state_sizes(lib):
+    assert lib.sr_gate_workspace_bytes(1024, 8, 32, 30) == 0
+    w = lib.sr_gate_workspace_bytes(1024, 8, 1024, 1024)
+    assert w > 1024 * 28 * 1024 * 2 and w % 256 == 0
+    assert lib.sr_gate_workspace_bytes(1024, 1, 1024, 1024) == 0
+    assert lib.sr_gate_host_arena_bytes(16, 8, 32, 10) >= 16 * 8 * 32 * 4
+    s = lib.sr_incr_state_bytes(65536, 8, 30)
+    assert s >= 65536 * (8 * 4 + 8 * 32 * 4 + 28 * 16) and s % 256 == 0
+    assert lib.sr_incr_state_bytes(10, 8, 33) == 0
+    assert lib.sr_incr_state_bytes(10, 1, 30) == 0
+
+
+def test_incremental_and_advantage_reject_bad_arguments(lib):
+    fake = 1 << 20
+    assert lib.sr_incr_init(None, 1 << 20, 4, 8, 30, None) == binding.SR_ERR_NULL
+    assert lib.sr_incr_init(fake, 1 << 20, 4, 8, 0, None) == binding.SR_ERR_BAD_K
+    assert lib.sr_incr_init(fake, 1 << 20, 4, 8, 33, None) == binding.SR_ERR_BAD_K
+    assert lib.sr_incr_init(fake, 1 << 20, 4, 40, 30, None) == binding.SR_ERR_BAD_N
+    assert lib.sr_incr_init(fake, 16, 4, 8, 30, None) == binding.SR_ERR_STATE_SIZE
+    step = lib.sr_gate_step_incremental
+    assert step(None, 1 << 20, fake, 4, 8, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_NULL
+    assert step(fake, 1 << 20, None, 4, 8, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_NULL
+    assert step(fake, 1 << 20, fake, 4, 8, 0.12, 7, None, None, None, fake, None, None) == binding.SR_ERR_BAD_MODE
+    assert step(fake, 16, fake, 4, 8, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_STATE_SIZE
+    adv = lib.sr_grpo_advantage
+    assert adv(None, None, 4, 8, 1e-6, fake, None, None) == binding.SR_ERR_NULL
+    assert adv(fake, None, 4, 1, 1e-6, fake, None, None) == binding.SR_ERR_BAD_N
+    assert adv(None, None, 0, 8, 1e-6, None, None, None) == binding.SR_OK
+    assert lib.sr_probe_int32(0, 1, 1, 32, None, None) == binding.SR_ERR_NULL
+    assert lib.sr_probe_int32_ops(10, 4, 128) == 10 * 16 * 8 * 4 * 128
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libsr_gate.so")
+    with pytest.raises(binding.SrError):
+        binding.sr_version()
+
+
+def test_shard_groups_partitions_exactly():
+    for G in (0, 1, 7, 512, 65536):
+        for W in (1, 2, 3, 8):
+            spans = [sr.shard_groups(G, W, r) for r in range(W)]
+            assert spans[0][0] == 0 and spans[-1][1] == G
+            for (a, b), (c, d) in zip(spans, spans[1:]):
+                assert b == c
+            sizes = [b - a for a, b in spans]
+            assert max(sizes) - min(sizes) <= 1

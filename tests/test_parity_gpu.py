@@ -1,0 +1,255 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI.
+
+Integer outputs (pair distances, pair sums, stop masks) and the fp64 d_K must be
+bit-identical; fp32 advantages must agree to 1e-6 relative (exact zeros exactly)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2605_05802_b200 as sr
+from paper_2605_05802_b200 import workloads as W
+
+from helpers import IncrementalGate, advantage_gpu, assert_gate_matches, gate_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_workload(w, thresholds=None):
+    for thr in (thresholds or [w.threshold]):
+        want = oracle.gate(w.seqs, w.lens, w.K, thr, w.norm_mode, threads=8)
+        got = gate_gpu(w.seqs, w.lens, w.K, thr, w.norm_mode)
+        assert_gate_matches(got, want, f"{w.name} thr={thr}")
+    return want
+
+
+def test_c1_tiny_both_threshold_readings():
+    want = _check_workload(W.tiny_gate(raw_threshold=True))
+    assert 0 < want[3].sum() < 16
+    _check_workload(W.tiny_gate(raw_threshold=False))
+
+
+def test_c2_agent_ragged_lengths():
+    _check_workload(W.agent_gate(K=15), [0.12, 0.5])
+    _check_workload(W.agent_gate(K=30), [0.12, 0.5])
+    w = W.agent_gate(K=15)
+    got = gate_gpu(w.seqs, w.lens, w.K, 0.5, want_pair_dist=False)      # optional output omitted
+    want = oracle.gate(w.seqs, w.lens, w.K, 0.5)
+    assert_gate_matches(got, want, "C2 no pair_dist")
+
+
+def test_c3_large_group_n16():
+    want = _check_workload(W.large_group_gate(), [0.12, 0.09])
+    assert 0 < want[3].sum() < 4096
+
+
+def test_c4_token_level_small_slice_every_element():
+    w = W.token_gate(n_groups=24)
+    _check_workload(w, [0.12, 0.6])
+
+
+def test_c4_token_level_full_size():
+    w = W.token_gate()
+    want = oracle.gate(w.seqs, w.lens, w.K, 0.5, w.norm_mode, threads=8)
+    got = gate_gpu(w.seqs, w.lens, w.K, 0.5, w.norm_mode)
+    assert_gate_matches(got, want, "C4 full")
+    assert 0 < want[3].sum() < 1024
+
+
+def test_multiword_repeated_symbols_and_ragged_tails():
+    rng = np.random.default_rng(17)
+    for vocab, lo, hi, stride in [(3, 33, 200, 200), (40, 1, 130, 132), (1000, 90, 700, 704),
+                                  (7, 1000, 1024, 1024), (100000, 33, 65, 68)]:
+        G, N = 6, 5
+        seqs = rng.integers(0, vocab, size=(G, N, stride)).astype(np.int32)
+        lens = rng.integers(lo, hi + 1, size=(G, N)).astype(np.int32)
+        lens[0, 0] = 0
+        lens[1, :] = hi
+        want = oracle.gate(seqs, lens, stride, 0.5, threads=8)
+        got = gate_gpu(seqs, lens, stride, 0.5)
+        assert_gate_matches(got, want, f"multi vocab={vocab}")
+        K = (lo + hi) // 2                         # prefix truncation inside the multi-word path
+        if K > 32:
+            want = oracle.gate(seqs, lens, K, 0.5, threads=8)
+            got = gate_gpu(seqs, lens, K, 0.5)
+            assert_gate_matches(got, want, f"multi vocab={vocab} K={K}")
+
+
+@pytest.mark.parametrize("N", [2, 3, 7, 8, 16, 32])
+def test_group_sizes(N):
+    rng = np.random.default_rng(N)
+    for stride, K in [(32, 30), (32, 32), (8, 5), (160, 150)]:
+        G = 11
+        seqs = rng.integers(0, 6, size=(G, N, stride)).astype(np.int32)
+        lens = rng.integers(0, stride + 1, size=(G, N)).astype(np.int32)
+        want = oracle.gate(seqs, lens, K, 0.4, threads=8)
+        got = gate_gpu(seqs, lens, K, 0.4)
+        assert_gate_matches(got, want, f"N={N} K={K}")
+
+
+def test_single_word_edges():
+    rng = np.random.default_rng(1)
+    # K = 0, K = 1, K = 31, K = 32 (top bit of the word), lens NULL, extreme IDs
+    for K in (0, 1, 31, 32):
+        seqs = rng.integers(0, 3, size=(9, 8, 32)).astype(np.int32)
+        seqs[0] = np.iinfo(np.int32).max
+        seqs[1, ::2] = np.iinfo(np.int32).min
+        seqs[2] = -1
+        for lens in (None, rng.integers(0, 33, size=(9, 8)).astype(np.int32)):
+            want = oracle.gate(seqs, lens, K, 0.3)
+            got = gate_gpu(seqs, lens, K, 0.3)
+            assert_gate_matches(got, want, f"K={K}")
+    # identical group -> d_K = 0 exactly; disjoint equal-length group -> d_K = 1 exactly
+    seqs = np.zeros((2, 8, 32), dtype=np.int32)
+    seqs[0] = np.arange(32)
+    seqs[1] = np.arange(8 * 32).reshape(8, 32)
+    _, _, mean, stop = gate_gpu(seqs, None, 30, 0.12)
+    assert mean.tolist() == [0.0, 1.0] and stop.tolist() == [1, 0]
+
+
+def test_threshold_is_strict_and_modes():
+    seqs = np.zeros((1, 2, 4), dtype=np.int32)
+    seqs[0, 0] = [1, 2, 3, 4]
+    seqs[0, 1] = [1, 2, 3, 5]
+    _, _, mean, stop = gate_gpu(seqs, None, 4, 0.25)
+    assert mean[0] == 0.25 and stop[0] == 0
+    _, _, _, stop = gate_gpu(seqs, None, 4, np.nextafter(0.25, 1.0))
+    assert stop[0] == 1
+    _, ps, mean, _ = gate_gpu(seqs, None, 4, 0.25, sr.SR_NORM_NONE)
+    assert ps[0] == 1 and mean[0] == 1.0
+
+
+def test_negative_lengths_are_clamped_and_flagged():
+    rng = np.random.default_rng(6)
+    for stride in (32, 96):
+        seqs = rng.integers(0, 4, size=(5, 4, stride)).astype(np.int32)
+        lens = rng.integers(1, stride, size=(5, 4)).astype(np.int32)
+        lens[2, 1] = -5
+        st = []
+        got = gate_gpu(seqs, lens, stride, 0.3, status=st)
+        want = oracle.gate(seqs, np.maximum(lens, 0), stride, 0.3)
+        assert_gate_matches(got, want, "neg len")
+        assert st[0] & sr.SR_STATUS_NEG_LEN
+
+
+def test_host_buffer_entry_point():
+    w = W.agent_gate(K=15)
+    for wl in (w, W.token_gate(n_groups=8)):
+        G, N, stride = wl.seqs.shape
+        P = N * (N - 1) // 2
+        h_seqs = torch.from_numpy(wl.seqs).pin_memory()
+        h_lens = torch.from_numpy(wl.lens).pin_memory()
+        pd = torch.empty((G, P), dtype=torch.int32).pin_memory()
+        ps = torch.empty((G,), dtype=torch.int32).pin_memory()
+        mean = torch.empty((G,), dtype=torch.float64).pin_memory()
+        stop = torch.empty((G,), dtype=torch.uint8).pin_memory()
+        arena = torch.empty(sr.sr_gate_host_arena_bytes(G, N, stride, wl.K), dtype=torch.uint8, device="cuda:0")
+        sr.sr_gate_host(h_seqs, h_lens, wl.K, 0.5, pair_dist=pd, pair_sum=ps, mean=mean, stop=stop, arena=arena)
+        torch.cuda.synchronize()
+        want = oracle.gate(wl.seqs, wl.lens, wl.K, 0.5, threads=8)
+        assert_gate_matches((pd.numpy(), ps.numpy(), mean.numpy(), stop.numpy()), want, "host " + wl.name)
+
+
+# ------------------------------------------------------------------ incremental
+def _check_stream(s, G=None):
+    actions = s.actions if G is None else s.actions[:, :G]
+    inc = IncrementalGate(actions.shape[1], actions.shape[2], max_steps=actions.shape[0])
+    for t, opd, ops, omean, ostop in oracle.gate_stream(actions, s.threshold, s.norm_mode, threads=8):
+        got = inc.step(actions[t - 1], s.threshold, s.norm_mode)
+        assert_gate_matches(got, (opd, ops, omean, ostop), f"{s.name} step {t}")
+    assert int(inc.status.item()) == 0
+    return inc
+
+
+def test_c5_incremental_equals_recompute_every_step():
+    _check_stream(W.streaming_gate(n_groups=2048))
+
+
+def test_c5_incremental_ragged_termination():
+    _check_stream(W.streaming_gate(n_groups=1024, ragged=True))
+
+
+def test_incremental_full_size_final_step():
+    s = W.streaming_gate()
+    inc = IncrementalGate(s.n_groups, s.N, max_steps=s.steps)
+    for t in range(s.steps):
+        got = inc.step(s.actions[t], s.threshold, s.norm_mode)
+        if t in (0, 14, 29):
+            seqs, lens = W.stream_prefix(s.actions, t + 1)
+            want = oracle.gate(seqs, lens, 32, s.threshold, s.norm_mode, threads=8)
+            assert_gate_matches(got, want, f"C5 full step {t + 1}")
+
+
+def test_incremental_other_group_sizes_overflow_and_snapshot():
+    rng = np.random.default_rng(12)
+    for N in (2, 5, 16):
+        G, steps = 37, 32
+        actions = rng.integers(0, 4, size=(steps, G, N)).astype(np.int32)
+        actions[rng.random(actions.shape) < 0.2] = sr.SR_NO_ACTION
+        inc = IncrementalGate(G, N, max_steps=32)
+        snap = None
+        for t, opd, ops, omean, ostop in oracle.gate_stream(actions, 0.4, 0):
+            got = inc.step(actions[t - 1], 0.4)
+            assert_gate_matches(got, (opd, ops, omean, ostop), f"N={N} step {t}")
+            if t == 15:
+                snap = inc.state.clone()
+        # restore the snapshot into a fresh buffer and replay: identical results
+        inc2 = IncrementalGate(G, N, max_steps=32)
+        inc2.state.copy_(snap)
+        for t in range(15, steps):
+            got2 = inc2.step(actions[t], 0.4)
+        assert_gate_matches(got2, got, "snapshot replay")
+    # a 33rd action is ignored and flagged
+    inc = IncrementalGate(3, 4, max_steps=4)
+    a = np.ones((3, 4), dtype=np.int32)
+    for _ in range(4):
+        before = inc.step(a, 0.4)
+    after = inc.step(a, 0.4)
+    assert_gate_matches(after, before, "overflow ignored")
+    assert int(inc.status.item()) & sr.SR_STATUS_STEP_OVERFLOW
+    # state formatted for other sizes is refused
+    inc.status.zero_()
+    bad = torch.from_numpy(np.ones((2, 4), dtype=np.int32)).cuda()
+    sr.sr_gate_step_incremental(inc.state, bad, 0.4, stop=inc.stop[:2], status=inc.status)
+    torch.cuda.synchronize()
+    assert int(inc.status.item()) & sr.SR_STATUS_BAD_STATE
+
+
+# -------------------------------------------------------------------- advantages
+def _check_adv(rewards, drop=None, eps=1e-6):
+    adv, zv = advantage_gpu(rewards, drop, eps)
+    oadv, ozv = oracle.advantage(rewards, drop, eps)
+    assert np.array_equal(zv, ozv)
+    zero = oadv == 0
+    assert np.array_equal(adv == 0, zero) and not np.signbit(adv[zero]).any()
+    nan = np.isnan(oadv)
+    assert np.array_equal(np.isnan(adv), nan)
+    ok = ~zero & ~nan
+    assert np.all(np.abs(adv[ok] - oadv[ok]) <= 1e-6 * np.abs(oadv[ok]))
+    return adv, zv
+
+
+def test_advantages_on_every_config():
+    for w in (W.tiny_gate(), W.agent_gate(), W.large_group_gate(), W.token_gate(n_groups=1024)):
+        _, zv = _check_adv(w.rewards)
+    s = W.streaming_gate()
+    _, zv = _check_adv(s.rewards)
+    assert 0 < zv.sum() < s.n_groups
+    drop = (np.arange(s.n_groups) % 3 == 0).astype(np.uint8)
+    adv, _ = _check_adv(s.rewards, drop)
+    assert (adv[drop == 1] == 0).all()
+
+
+def test_advantage_edges():
+    rng = np.random.default_rng(3)
+    for N in (2, 3, 5, 8, 16, 31, 32):
+        r = rng.random((257, N)).astype(np.float32)
+        r[0] = 0.3
+        r[1] = -0.0
+        r[1, 0] = 0.0
+        r[2, 0] = np.nan
+        r[3] = np.float32(1e30)
+        r[4, : N // 2] = 1.0
+        r[4, N // 2:] = 0.0
+        for eps in (1e-6, 0.0):
+            _check_adv(r, None, eps)
