@@ -99,9 +99,12 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
     }
     __syncthreads();
     for (int g = 0; g < ng; ++g) {
-        const int words = N * s_cnt[g];
+        const int cnt = s_cnt[g];
         uint32_t* peq = s_peq + (size_t)g * N * L.dmax;
-        for (int e = tid; e < words; e += nthr) peq[e] = 0u;
+        for (int e = tid; e < N * cnt; e += nthr) {
+            const int i = e / cnt;
+            peq[i * L.dmax + (e - i * cnt)] = 0u;
+        }
     }
     __syncthreads();
     for (int e = tid; e < ng * per_group; e += nthr) {
