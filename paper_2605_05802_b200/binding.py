@@ -42,6 +42,8 @@ _SIGNATURES = {
     "sr_gate_step_incremental": (ctypes.c_int, [_vp, _sz, _vp, _i32, _i32, _f64, _i32, _vp, _vp, _vp,
                                                 _vp, _vp, _vp]),
     "sr_grpo_advantage": (ctypes.c_int, [_vp, _vp, _i32, _i32, _f32, _vp, _vp, _vp]),
+    "sr_gate_stages": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
+                                      _vp, _vp, _sz, _vp, _vp]),
     "sr_probe_int32": (ctypes.c_int, [_i32, _i32, _i32, _i32, _vp, _vp]),
     "sr_probe_int32_ops": (ctypes.c_uint64, [_i32, _i32, _i32]),
 }
@@ -119,6 +121,20 @@ def sr_gate(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, threshold:
                           _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
                           _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(workspace),
                           ws_bytes, _stream(stream)))
+
+
+def sr_gate_stages(seqs, lens, K, threshold, norm_mode=SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None,
+                   mean=None, stop=None, status=None, workspace=None, stream=None, events=None) -> None:
+    """sr_gate that also records five torch.cuda.Event (created with
+    enable_timing=True and recorded once beforehand) at the pipeline's stage boundaries."""
+    G, N, stride = seqs.shape
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    handles = (ctypes.c_void_p * 5)(*[e.cuda_event for e in events])
+    _check(load().sr_gate_stages(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
+                                 float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
+                                 _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
+                                 _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(workspace),
+                                 ws_bytes, _stream(stream), handles))
 
 
 def sr_gate_host_arena_bytes(n_groups: int, N: int, stride: int, K: int) -> int:

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include "common.cuh"
+#include "sr_probe.h"
 
 namespace sr {
 
@@ -93,6 +94,35 @@ int sr_gate(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t 
             return SR_ERR_WORKSPACE;
     }
     return launch_gate_multi(a, workspace, workspace_bytes, s);
+}
+
+int sr_gate_stages(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                   int32_t stride, int32_t K, double threshold, int32_t norm_mode,
+                   int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                   int32_t* status, void* workspace, size_t workspace_bytes, void* stream,
+                   void* const* events) {
+    if (events == nullptr) return SR_ERR_NULL;
+    for (int k = 0; k < 5; ++k)
+        if (events[k] == nullptr) return SR_ERR_NULL;
+    const int rc = check_gate_args(seqs, n_groups, N, stride, K, norm_mode, stop);
+    if (rc != SR_OK) return rc;
+    GateArgs a{seqs, lens, n_groups, N, stride, K, threshold, norm_mode,
+               pair_dist, pair_sum, mean, stop, status};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaEvent_t ev[5];
+    for (int k = 0; k < 5; ++k) ev[k] = static_cast<cudaEvent_t>(events[k]);
+    if (K <= 32 || n_groups == 0) {
+        SR_CUDA_TRY(cudaEventRecord(ev[0], s));
+        const int r = (K <= 32) ? launch_gate_single(a, s) : SR_OK;
+        if (r != SR_OK) return r;
+        for (int k = 1; k < 5; ++k) SR_CUDA_TRY(cudaEventRecord(ev[k], s));
+        return SR_OK;
+    }
+    const size_t need = gate_multi_workspace_bytes(n_groups, N, stride, K);
+    if (workspace == nullptr || workspace_bytes < need ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
+        return SR_ERR_WORKSPACE;
+    return launch_gate_multi(a, workspace, workspace_bytes, s, ev);
 }
 
 size_t sr_gate_host_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K) {

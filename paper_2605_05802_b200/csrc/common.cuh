@@ -77,7 +77,10 @@ size_t align_up(size_t x, size_t a);
 int launch_gate_single(const GateArgs& a, cudaStream_t s);
 // gate_multi.cu: prefixes of up to SR_MAX_K symbols, blocked multi-word.
 size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
-int launch_gate_multi(const GateArgs& a, void* ws, size_t ws_bytes, cudaStream_t s);
+// `ev`: NULL, or 5 events recorded before prep / after prep / after scan+scatter /
+// after dp / after finish.
+int launch_gate_multi(const GateArgs& a, void* ws, size_t ws_bytes, cudaStream_t s,
+                      const cudaEvent_t* ev = nullptr);
 // incremental.cu
 size_t incr_state_bytes(int32_t n_groups, int32_t N, int32_t max_steps);
 int launch_incr_init(void* state, size_t bytes, int32_t n_groups, int32_t N, int32_t max_steps,

@@ -393,7 +393,8 @@ size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, i
     return multi_layout(n_groups, N, K).total;
 }
 
-int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_t s) {
+int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_t s,
+                      const cudaEvent_t* ev) {
     if (a.n_groups == 0) return SR_OK;
     const MultiWs W = multi_layout(a.n_groups, a.N, a.K);
     if (ws_ == nullptr || ws_bytes < W.total || (reinterpret_cast<uintptr_t>(ws_) & 255) != 0)
@@ -412,15 +413,18 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     while ((1 << (32 - hshift)) < hslots) --hshift;
     const int prep_smem = W.pitch * 4 + hslots * 8 + W.pitch * 2;
 
+    if (ev) SR_CUDA_TRY(cudaEventRecord(ev[0], s));
     SR_CUDA_TRY(cudaMemsetAsync(ctl->hist, 0, sizeof(ctl->hist), s));
     multi_prep_kernel<<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, hshift, dist);
     SR_LAUNCH_CHECK("multi_prep_kernel");
+    if (ev) SR_CUDA_TRY(cudaEventRecord(ev[1], s));
     multi_scan_kernel<<<1, kNumBins, 0, s>>>(ctl);
     SR_LAUNCH_CHECK("multi_scan_kernel");
     multi_scatter_kernel<<<(n_pairs + 255) / 256, 256, 0, s>>>(
         reinterpret_cast<const PairDesc*>(ws + W.off_desc),
         reinterpret_cast<int32_t*>(ws + W.off_order), ctl, n_pairs);
     SR_LAUNCH_CHECK("multi_scatter_kernel");
+    if (ev) SR_CUDA_TRY(cudaEventRecord(ev[2], s));
     int dev = 0, sms = 0;
     SR_CUDA_TRY(cudaGetDevice(&dev));
     SR_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
@@ -431,8 +435,10 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     if (blocks < 1) blocks = 1;
     multi_dp_kernel<<<blocks, kDpWarpsPerCta * 32, 0, s>>>(ws, W, dist);
     SR_LAUNCH_CHECK("multi_dp_kernel");
+    if (ev) SR_CUDA_TRY(cudaEventRecord(ev[3], s));
     multi_finish_kernel<<<(a.n_groups + 127) / 128, 128, 0, s>>>(a, dist);
     SR_LAUNCH_CHECK("multi_finish_kernel");
+    if (ev) SR_CUDA_TRY(cudaEventRecord(ev[4], s));
     return SR_OK;
 }
 
