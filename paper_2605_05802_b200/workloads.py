@@ -264,6 +264,20 @@ def dp_cells(lens: np.ndarray, K: int) -> int:
     return int(((s1 * s1 - s2) // 2).sum())
 
 
+def word_columns(lens: np.ndarray, K: int) -> int:
+    """Work units of the bit-vector method: the sum over unordered pairs of
+    (text columns) x (32-row blocks of the pattern), taking for every pair the
+    cheaper of the two orientations.  Used only to express roofline fractions."""
+    m = np.minimum(np.maximum(lens.astype(np.int64), 0), K)
+    w = (m + 31) // 32
+    total = 0
+    N = lens.shape[1]
+    for i in range(N):
+        for j in range(i + 1, N):
+            total += int(np.minimum(m[:, i] * w[:, j], m[:, j] * w[:, i]).sum())
+    return total
+
+
 def all_gate_configs() -> List[GateWorkload]:
     return [tiny_gate(), tiny_gate(raw_threshold=False), agent_gate(K=15), agent_gate(K=30),
             large_group_gate(), token_gate()]
