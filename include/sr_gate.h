@@ -40,6 +40,7 @@ extern "C" {
 #define SR_ERR_WORKSPACE (-6)      /* workspace NULL, misaligned or too small */
 #define SR_ERR_CUDA (-7)           /* a CUDA call failed; see sr_last_cuda_error() */
 #define SR_ERR_BAD_MODE (-8)       /* unknown norm_mode */
+#define SR_ERR_SCRATCH_LIMIT (-9)  /* sr_gate_noalloc: problem needs more than the built-in scratch */
 
 /* limits */
 #define SR_MAX_N 32                /* rollouts per group */
@@ -114,6 +115,39 @@ int sr_gate_host(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int
                  int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
                  int32_t* status, void* arena, size_t arena_bytes, void* stream);
 size_t sr_gate_host_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
+
+/*
+ * sr_gate_noalloc -- sr_gate for callers that cannot allocate device memory.  (The
+ * paper has no counterpart: this is a deployment aid of this library.)
+ *
+ * Who needs it: a gate that runs inside someone else's process -- a rollout worker
+ * embedded in an inference engine that claimed its GPU memory at start-up, a trainer
+ * whose caching allocator owns the rest, a plug-in that is simply not allowed to
+ * call cudaMalloc.  There sr_gate's `workspace` has nowhere to come from.  This
+ * entry point takes the same inputs and outputs but no workspace: the multi-word
+ * path (K > 32) works in a fixed array of SR_NOALLOC_SCRATCH_BYTES that is part of
+ * the library's device image, so every GPU on which the library is used holds that
+ * much memory from load until the process exits.  It calls no allocation routine.
+ *
+ *   - Limit: sr_gate_workspace_bytes(n_groups, N, stride, K) must not exceed
+ *     SR_NOALLOC_SCRATCH_BYTES (also returned by sr_gate_noalloc_limit_bytes());
+ *     otherwise SR_ERR_SCRATCH_LIMIT, nothing enqueued.  As a guide, 64 groups of
+ *     N = 8 at K = 1024, or 1000 groups at K = 64, fit.  K <= 32 has no limit.
+ *   - The first call on each device looks up the array's device address (a
+ *     cudaGetSymbolAddress with that device current).  Make that first call during
+ *     set-up, before any stream capture is begun.
+ *   - All calls on a device share the one array.  It keeps whatever the last call
+ *     left; each call clears the counters it needs zeroed before using them.  Two
+ *     calls that can overlap on the device (different streams, no dependency) race
+ *     on it: serialise them, or use sr_gate with separate workspaces.
+ *   - Results are identical to sr_gate's.
+ */
+#define SR_NOALLOC_SCRATCH_BYTES (16u << 20)
+int sr_gate_noalloc(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                    int32_t stride, int32_t K, double threshold, int32_t norm_mode,
+                    int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                    int32_t* status, void* stream);
+size_t sr_gate_noalloc_limit_bytes(void);
 
 /*
  * Incremental gate: the gate re-evaluated after every environment step while

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(HERE, "libsr_gate.so")
 SR_OK = 0
 SR_ERR_NULL, SR_ERR_BAD_N, SR_ERR_BAD_K, SR_ERR_ALIGN = -1, -2, -3, -4
 SR_ERR_STATE_SIZE, SR_ERR_WORKSPACE, SR_ERR_CUDA, SR_ERR_BAD_MODE = -5, -6, -7, -8
+SR_ERR_SCRATCH_LIMIT = -9
 SR_NORM_MAXLEN, SR_NORM_NONE = 0, 1
 SR_NO_ACTION = -(2 ** 31)
 SR_STATUS_NEG_LEN, SR_STATUS_STEP_OVERFLOW, SR_STATUS_BAD_STATE = 1, 2, 4
@@ -33,6 +34,9 @@ _SIGNATURES = {
     "sr_last_cuda_error": (ctypes.c_char_p, []),
     "sr_gate": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp, _vp,
                                _vp, _sz, _vp]),
+    "sr_gate_noalloc": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
+                                       _vp, _vp]),
+    "sr_gate_noalloc_limit_bytes": (_sz, []),
     "sr_gate_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "sr_gate_host": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
                                     _vp, _vp, _sz, _vp]),
@@ -121,6 +125,26 @@ def sr_gate(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, threshold:
                           _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
                           _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(workspace),
                           ws_bytes, _stream(stream)))
+
+
+def sr_gate_noalloc_limit_bytes() -> int:
+    return int(load().sr_gate_noalloc_limit_bytes())
+
+
+def sr_gate_noalloc(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, threshold: float,
+                    norm_mode: int = SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None, mean=None,
+                    stop=None, status=None, stream=None) -> None:
+    """sr_gate without a workspace argument, for code that may not allocate on the
+    device (it runs inside a process whose GPU memory is already spoken for).  The
+    scratch is a fixed array inside the library; problems whose scratch need exceeds
+    sr_gate_noalloc_limit_bytes() are refused with SR_ERR_SCRATCH_LIMIT.  Calls that
+    may overlap on the device must be serialised by the caller."""
+    G, N, stride = seqs.shape
+    _check(load().sr_gate_noalloc(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
+                                  float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
+                                  _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
+                                  _ptr(stop, torch.uint8), _ptr(status, torch.int32),
+                                  _stream(stream)))
 
 
 def sr_gate_stages(seqs, lens, K, threshold, norm_mode=SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None,

@@ -12,7 +12,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsr_gate.so")
-SOURCES = ["api.cu", "gate_single.cu", "gate_multi.cu", "incremental.cu", "advantage.cu", "probe.cu"]
+SOURCES = ["api.cu", "gate_single.cu", "gate_multi.cu", "incremental.cu", "advantage.cu", "probe.cu",
+           "gate_noalloc.cu"]
 
 
 def _stale() -> bool:

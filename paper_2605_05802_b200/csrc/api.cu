@@ -65,6 +65,7 @@ const char* sr_strerror(int code) {
         case SR_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case SR_ERR_CUDA: return "a CUDA call failed (see sr_last_cuda_error)";
         case SR_ERR_BAD_MODE: return "unknown norm_mode";
+        case SR_ERR_SCRATCH_LIMIT: return "problem needs more scratch than sr_gate_noalloc's built-in array";
         default: return "unknown error code";
     }
 }
