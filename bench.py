@@ -159,6 +159,8 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--groups", type=int, default=1024,
+                    help="groups per GPU of the token-level workload (1024 = the benchmark configuration)")
     ap.add_argument("--no-extras", action="store_true", help="skip the per-config side measurements")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -205,7 +207,7 @@ def main():
         return [a.elapsed_time(b) for a, b in evs]
 
     # ------------------------------------------------------------ headline workload
-    w = W.token_gate(seed=3 + 1000 * rank)      # every rank gates its own 1024 groups
+    w = W.token_gate(seed=3 + 1000 * rank, n_groups=args.groups)      # every rank gates its own 1024 groups
     G, N, stride, K = w.n_groups, w.N, w.stride, w.K
     P = N * (N - 1) // 2
     cells = W.dp_cells(w.lens, K)
@@ -300,7 +302,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": "C4-token: 1024 groups x N=8 rollouts per GPU, token prefixes U{256..1024}, "
+        "config": {"workload": f"C4-token: {args.groups} groups x N=8 rollouts per GPU, token prefixes U{256..1024}, "
                                "vocab 151936, K=1024, d_L=0.12; gate + advantages",
                    "groups_per_gpu": G, "pairs_per_group": P, "dp_cells_per_gpu": cells,
                    "l2": "flushed before every step (256 MiB write)", "parallelism": f"groups sharded x{world}, no collective"},
