@@ -302,7 +302,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-        "config": {"workload": f"C4-token: {args.groups} groups x N=8 rollouts per GPU, token prefixes U{256..1024}, "
+        "config": {"workload": f"C4-token: {args.groups} groups x N=8 rollouts per GPU, token prefixes U[256..1024], "
                                "vocab 151936, K=1024, d_L=0.12; gate + advantages",
                    "groups_per_gpu": G, "pairs_per_group": P, "dp_cells_per_gpu": cells,
                    "l2": "flushed before every step (256 MiB write)", "parallelism": f"groups sharded x{world}, no collective"},
