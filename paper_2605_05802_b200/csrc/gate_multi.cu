@@ -10,7 +10,7 @@
 //   prep     one CTA per (group, pattern rollout): hashes the pattern's symbols
 //            in shared memory, then translates every text paired with it into a
 //            "loc" stream: for text column c the position of the column's symbol in
-//            the pattern (0xFFFF: absent; bit 15 set: several occurrences, walk
+//            the pattern (0x7FFF: absent; bit 15 set: several occurrences, walk
 //            the pattern's chain).  A block's match word is then just
 //            1 << (loc - first_row_of_block), no table lookup.  Also bins the pairs
 //            by (team shape, text length).
@@ -36,7 +36,7 @@ constexpr int kPrepThreads = 256;
 constexpr int kNumClasses = 16;     // class = log2(T) * 4 + (R - 1)
 constexpr int kLenBuckets = 64;     // text length / 16
 constexpr int kNumBins = kNumClasses * kLenBuckets;
-constexpr uint32_t kLocNone = 0xFFFFu;
+constexpr uint32_t kLocNone = 0x7FFFu;    // bit 15 clear, far above any row: shifts to 0
 constexpr uint32_t kLocMulti = 0x8000u;
 constexpr uint32_t kChainEnd = 0xFFFFu;
 constexpr int kDpWarpsPerCta = 4;
@@ -247,6 +247,52 @@ __device__ __forceinline__ uint32_t shl_clamp(uint32_t v, uint32_t s) {
     return r;
 }
 
+// One bit-vector column step over the R blocks a lane owns.  `loc` is the column's
+// entry of the match stream, (inP, inM) the pre-shift horizontal delta words of the
+// block above (only their top bits matter); returns this lane's last block's words in
+// (inP, inM).
+template <int R>
+__device__ __forceinline__ void column_step(uint32_t loc, uint32_t rowbase, int m,
+                                            const uint16_t* __restrict__ nxt,
+                                            uint32_t (&Pv)[R], uint32_t (&Mv)[R],
+                                            uint32_t& inP, uint32_t& inM) {
+    const uint32_t d0 = loc - rowbase;
+    uint32_t Eq[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) Eq[r] = shl_clamp(1u, d0 - 32u * r);
+    if (loc & kLocMulti) {          // several occurrences in the pattern: walk the chain
+        uint32_t p = loc & 0x7FFFu;
+        for (int hop = 0; hop < SR_MAX_K && p < (uint32_t)m; ++hop) {   // chain ends at 0xFFFF
+            const uint32_t dd = p - rowbase;
+#pragma unroll
+            for (int r = 0; r < R; ++r) Eq[r] |= shl_clamp(1u, dd - 32u * r);
+            p = __ldg(nxt + p);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const uint32_t pv = Pv[r], mv = Mv[r];
+        const uint32_t Xv = Eq[r] | mv;
+        const uint32_t Eh = Eq[r] | (inM >> 31);
+        const uint32_t Xh = (((Eh & pv) + pv) ^ pv) | Eh;
+        const uint32_t Ph = mv | ~(Xh | pv);
+        const uint32_t Mh = pv & Xh;
+        const uint32_t Phs = __funnelshift_l(inP, Ph, 1);
+        const uint32_t Mhs = __funnelshift_l(inM, Mh, 1);
+        Pv[r] = Mhs | ~(Xv | Phs);
+        Mv[r] = Phs & Xv;
+        inP = Ph;
+        inM = Mh;
+    }
+}
+
+// A warp task: 32/T teams of T lanes, one pair per team, lane l of a team holding
+// rows [32*R*l, 32*R*(l+1)) of the pattern.  Lanes are skewed by one QUAD of text
+// columns: in iteration j lane l works on columns 4(j-l) .. 4(j-l)+3.  The four
+// columns are unrolled, so (a) a lane fetches its four stream entries with one
+// 8-byte load, one iteration ahead, (b) the delta words a lane needs from the lane
+// above were produced a whole iteration earlier, so the shuffles never wait, and (c)
+// the blocks of consecutive columns overlap in the pipeline.
 template <int R>
 __device__ __forceinline__ void dp_task(int tlog, int pos, bool valid, const PairDesc* descs,
                                         const int32_t* order, const uint16_t* locs,
@@ -255,81 +301,62 @@ __device__ __forceinline__ void dp_task(int tlog, int pos, bool valid, const Pai
     const int T = 1 << tlog;
     const int lt = lane & (T - 1);
     int idx = 0, m = 0, n = 0;
-    const uint16_t* loc = locs;
+    const uint2* loc4 = reinterpret_cast<const uint2*>(locs);
     const uint16_t* nxt = nexts;
     if (valid) {
         idx = order[pos];
         const PairDesc d = descs[idx];
         m = (int)(d.mn & 0xFFFFu);
         n = (int)(d.mn >> 16);
-        loc = locs + (size_t)idx * pitch;
+        loc4 = reinterpret_cast<const uint2*>(locs + (size_t)idx * pitch);   // rows are 16-byte aligned
         nxt = nexts + (size_t)d.pat_row * pitch;
     }
-    const int rowbase = lt * R * 32;
-    int nsteps = valid ? n + T - 1 : 0;
-    nsteps = __reduce_max_sync(0xFFFFFFFFu, nsteps);
+    const uint32_t rowbase = (uint32_t)(lt * R * 32);
+    const int nq = (n + 3) >> 2;                       // quads of text columns
+    int iters = valid ? nq + T - 1 : 0;
+    iters = __reduce_max_sync(0xFFFFFFFFu, iters);
+    const bool top = lt == 0;
 
     uint32_t Pv[R], Mv[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) { Pv[r] = 0xFFFFFFFFu; Mv[r] = 0u; }
-    uint32_t lastP = 0u, lastM = 0u;
-    uint32_t loc_nxt = (valid && lt == 0) ? (uint32_t)__ldg(loc) : kLocNone;
+    uint32_t outP[4] = {0u, 0u, 0u, 0u}, outM[4] = {0u, 0u, 0u, 0u};
+    const uint2 none = make_uint2(kLocNone | (kLocNone << 16), kLocNone | (kLocNone << 16));
+    uint2 q_next = (valid && top) ? __ldg(loc4) : none;
 
-    for (int s = 0; s < nsteps; ++s) {
-        const int c = s - lt;
-        const bool active = valid && c >= 0 && c < n;
-        const uint32_t loc_now = loc_nxt;
-        {
-            const int cn = c + 1;
-            loc_nxt = (valid && cn >= 0 && cn < n) ? (uint32_t)__ldg(loc + cn) : kLocNone;
+    for (int j = 0; j < iters; ++j) {
+        const int qi = j - lt;
+        const bool active = valid && qi >= 0 && qi < nq;
+        const uint2 q = q_next;
+        q_next = (valid && qi + 1 >= 0 && qi + 1 < nq) ? __ldg(loc4 + qi + 1) : none;
+        // delta words leaving the lane above for this quad (it worked on it last iteration)
+        uint32_t inP[4], inM[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            inP[u] = __shfl_up_sync(0xFFFFFFFFu, outP[u], 1);
+            inM[u] = __shfl_up_sync(0xFFFFFFFFu, outM[u], 1);
+            if (top) { inP[u] = 0x80000000u; inM[u] = 0u; }   // row 0: D[0][c] - D[0][c-1] = +1
         }
-        // horizontal deltas leaving the lane above (its previous step = this column)
-        uint32_t inP = __shfl_up_sync(0xFFFFFFFFu, lastP, 1);
-        uint32_t inM = __shfl_up_sync(0xFFFFFFFFu, lastM, 1);
-        if (lt == 0) { inP = 0x80000000u; inM = 0u; }      // row 0: D[0][c] - D[0][c-1] = +1
         if (active) {
-            const uint32_t d0 = loc_now - (uint32_t)rowbase;
-            uint32_t Eq[R];
+            const int left = n - 4 * qi;               // columns of this quad that exist (>= 1)
+            column_step<R>(q.x & 0xFFFFu, rowbase, m, nxt, Pv, Mv, inP[0], inM[0]);
+            if (left > 1) column_step<R>(q.x >> 16, rowbase, m, nxt, Pv, Mv, inP[1], inM[1]);
+            if (left > 2) column_step<R>(q.y & 0xFFFFu, rowbase, m, nxt, Pv, Mv, inP[2], inM[2]);
+            if (left > 3) column_step<R>(q.y >> 16, rowbase, m, nxt, Pv, Mv, inP[3], inM[3]);
 #pragma unroll
-            for (int r = 0; r < R; ++r) Eq[r] = shl_clamp(1u, d0 - 32u * r);
-            if (loc_now >= kLocMulti && loc_now != kLocNone) {
-                uint32_t p = loc_now & 0x7FFFu;
-                for (int hop = 0; hop < SR_MAX_K && p < (uint32_t)m; ++hop) {   // chain ends at 0xFFFF
-                    const uint32_t dd = p - (uint32_t)rowbase;
-#pragma unroll
-                    for (int r = 0; r < R; ++r) Eq[r] |= shl_clamp(1u, dd - 32u * r);
-                    p = __ldg(nxt + p);
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const uint32_t pv = Pv[r], mv = Mv[r];
-                const uint32_t Xv = Eq[r] | mv;
-                const uint32_t Eh = Eq[r] | (inM >> 31);
-                const uint32_t Xh = (((Eh & pv) + pv) ^ pv) | Eh;
-                const uint32_t Ph = mv | ~(Xh | pv);
-                const uint32_t Mh = pv & Xh;
-                const uint32_t Phs = __funnelshift_l(inP, Ph, 1);
-                const uint32_t Mhs = __funnelshift_l(inM, Mh, 1);
-                Pv[r] = Mhs | ~(Xv | Phs);
-                Mv[r] = Phs & Xv;
-                inP = Ph;
-                inM = Mh;
-            }
-            lastP = inP;
-            lastM = inM;
+            for (int u = 0; u < 4; ++u) { outP[u] = inP[u]; outM[u] = inM[u]; }
         }
     }
     // D[m][n] = n + (sum of the vertical deltas of the last column over rows 1..m)
     int part = 0;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        const int rows = min(max(m - (rowbase + 32 * r), 0), 32);
+        const int rows = min(max(m - (int)(rowbase + 32 * r), 0), 32);
         const uint32_t msk = low_mask(rows);
         part += __popc(Pv[r] & msk) - __popc(Mv[r] & msk);
     }
     for (int off = 1; off < T; off <<= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, off);
-    if (valid && lt == 0) dist_out[idx] = n + part;
+    if (valid && top) dist_out[idx] = n + part;
 }
 
 __global__ void __launch_bounds__(kDpWarpsPerCta * 32)
