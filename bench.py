@@ -260,7 +260,7 @@ def main():
                           workspace=ws, events=e5)
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
-    stage_ms = [statistics.mean(e5[k].elapsed_time(e5[k + 1]) for e5 in stage_evs) for k in range(4)]
+    stage_ms = [statistics.median(e5[k].elapsed_time(e5[k + 1]) for e5 in stage_evs) for k in range(4)]
     dp_ms = stage_ms[2]
 
     # ------------------------------------------------------------------ end to end

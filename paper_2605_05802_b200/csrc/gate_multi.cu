@@ -118,14 +118,30 @@ __device__ __forceinline__ int clamp_len(const int32_t* lens, size_t idx, int K,
 }
 
 // ------------------------------------------------------------------------ prep
+// Position (or chain head) of `sym` in the pattern hashed in shared memory.
+__device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, const int32_t* s_pat,
+                                                   const uint32_t* s_owner, const uint32_t* s_next,
+                                                   int hslots, int hshift) {
+    uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> hshift;
+    for (int probe = 0; probe < hslots; ++probe) {     // an empty slot always exists
+        const uint32_t o = s_owner[h];
+        if (o == 0u) break;
+        if (s_pat[o - 1u] == sym) {
+            const uint32_t first = o - 1u;
+            return s_next[first] == kChainEnd ? first : (kLocMulti | first);
+        }
+        h = (h + 1u) & (uint32_t)(hslots - 1);
+    }
+    return kLocNone;
+}
+
 __global__ void __launch_bounds__(kPrepThreads)
-multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots, int hshift,
-                  int32_t* dist_out) {
+multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int32_t* dist_out) {
     extern __shared__ __align__(16) unsigned char smem[];
     int32_t* s_pat = reinterpret_cast<int32_t*>(smem);                       // [pitch]
-    uint32_t* s_owner = reinterpret_cast<uint32_t*>(s_pat + W.pitch);        // [hslots]
-    uint32_t* s_head = s_owner + hslots;                                     // [hslots]
-    uint16_t* s_next = reinterpret_cast<uint16_t*>(s_head + hslots);         // [pitch]
+    uint32_t* s_owner = reinterpret_cast<uint32_t*>(s_pat + W.pitch);        // [hslots_max]
+    uint32_t* s_next = s_owner + hslots_max;                                 // [pitch]
+    __shared__ int s_txt[SR_MAX_N], s_len[SR_MAX_N], s_qstart[SR_MAX_N + 1], s_ntxt;
 
     const int N = a.N, K = a.K, P = pairs_of(N);
     const int g = blockIdx.x / N, i = blockIdx.x - g * N;
@@ -134,67 +150,84 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots, int hshi
     if (i >= M) return;                               // the last rollout of an even group is never a pattern
     bool neg = false;
     const int m = clamp_len(a.lens, (size_t)g * N + i, K, neg);
+    // the table holds at least twice as many slots as the pattern has symbols
+    int hslots = 64;
+    while (hslots < 2 * m) hslots <<= 1;
+    const int hshift = __clz(hslots) + 1;             // 32 - log2(hslots)
     const int32_t* pat = a.seqs + ((size_t)g * N + i) * a.stride;
-    for (int p = tid; p < m; p += kPrepThreads) s_pat[p] = __ldg(pat + p);
-    for (int h = tid; h < hslots; h += kPrepThreads) { s_owner[h] = 0u; s_head[h] = 0u; }
+    for (int q = tid; 4 * q < m; q += kPrepThreads) {   // rows are 16-byte aligned, stride % 4 == 0
+        reinterpret_cast<int4*>(s_pat)[q] = __ldg(reinterpret_cast<const int4*>(pat) + q);
+        reinterpret_cast<uint4*>(s_next)[q] = make_uint4(kChainEnd, kChainEnd, kChainEnd, kChainEnd);
+    }
+    for (int h = tid; h < hslots; h += kPrepThreads) s_owner[h] = 0u;
+    if (tid == 0) {                                   // the texts this pattern is paired with
+        int cnt = 0, quads = 0;
+        for (int j = 0; j < N; ++j) {
+            if (j == i) continue;
+            const int lo = min(i, j), hi = max(i, j);
+            if (first_is_pattern(lo, hi, N) != (lo == i)) continue;
+            const int n = clamp_len(a.lens, (size_t)g * N + j, K, neg);
+            s_txt[cnt] = j;
+            s_len[cnt] = n;
+            s_qstart[cnt] = quads;
+            quads += (m > 0) ? (n + 3) >> 2 : 0;
+            ++cnt;
+        }
+        s_qstart[cnt] = quads;
+        s_ntxt = cnt;
+    }
     __syncthreads();
-    // every position claims (or finds) the slot of its symbol and pushes itself on
-    // the slot's occurrence chain
+    // every position claims the slot of its symbol, or links itself behind the
+    // position that claimed it (the claimant heads the symbol's occurrence chain)
     for (int p = tid; p < m; p += kPrepThreads) {
         const int32_t sym = s_pat[p];
         uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> hshift;
-        // at least twice as many slots as symbols: a free or matching slot always
-        // exists; the trip count is bounded all the same
         for (int probe = 0; probe < hslots; ++probe) {
             uint32_t o = s_owner[h];
             if (o == 0u) o = atomicCAS(&s_owner[h], 0u, (uint32_t)p + 1u);
-            if (o == 0u || s_pat[o - 1u] == sym) break;
+            if (o == 0u) break;
+            if (s_pat[o - 1u] == sym) {
+                s_next[p] = atomicExch(&s_next[o - 1u], (uint32_t)p);
+                break;
+            }
             h = (h + 1u) & (uint32_t)(hslots - 1);
         }
-        const uint32_t prev = atomicExch(&s_head[h], (uint32_t)p + 1u);
-        s_next[p] = prev == 0u ? (uint16_t)kChainEnd : (uint16_t)(prev - 1u);
     }
     __syncthreads();
     uint16_t* g_next = reinterpret_cast<uint16_t*>(ws + W.off_next) + ((size_t)g * N + i) * W.pitch;
-    for (int p = tid; p < m; p += kPrepThreads) g_next[p] = s_next[p];
+    for (int p = tid; p < m; p += kPrepThreads) g_next[p] = (uint16_t)s_next[p];
 
     PairDesc* descs = reinterpret_cast<PairDesc*>(ws + W.off_desc);
     uint16_t* locs = reinterpret_cast<uint16_t*>(ws + W.off_loc);
     Ctl* ctl = reinterpret_cast<Ctl*>(ws + W.off_ctl);
-    int tlog, R;
-    team_shape(m, tlog, R);
-    for (int j = 0; j < N; ++j) {
-        if (j == i) continue;
+    const int ntxt = s_ntxt;
+    // match streams of all texts, four columns per thread and trip: one 16-byte load
+    // of symbols, four independent look-ups, one 8-byte store
+    const int total_quads = s_qstart[ntxt];
+    for (int item = tid; item < total_quads; item += kPrepThreads) {
+        int t = 0;
+        while (item >= s_qstart[t + 1]) ++t;
+        const int q = item - s_qstart[t];
+        const int j = s_txt[t];
         const int lo = min(i, j), hi = max(i, j);
-        if (first_is_pattern(lo, hi, N) != (lo == i)) continue;
-        const int n = clamp_len(a.lens, (size_t)g * N + j, K, neg);
+        const size_t idx = (size_t)g * P + pair_index(lo, hi, N);
+        const int4 sym = __ldg(reinterpret_cast<const int4*>(a.seqs + ((size_t)g * N + j) * a.stride) + q);
+        const uint32_t l0 = pattern_lookup(sym.x, s_pat, s_owner, s_next, hslots, hshift);
+        const uint32_t l1 = pattern_lookup(sym.y, s_pat, s_owner, s_next, hslots, hshift);
+        const uint32_t l2 = pattern_lookup(sym.z, s_pat, s_owner, s_next, hslots, hshift);
+        const uint32_t l3 = pattern_lookup(sym.w, s_pat, s_owner, s_next, hslots, hshift);
+        reinterpret_cast<uint2*>(locs + idx * W.pitch)[q] = make_uint2(l0 | (l1 << 16), l2 | (l3 << 16));
+    }
+    if (tid < ntxt) {                                 // descriptors, bins, trivial pairs
+        const int j = s_txt[tid], n = s_len[tid];
+        const int lo = min(i, j), hi = max(i, j);
         const size_t idx = (size_t)g * P + pair_index(lo, hi, N);
         if (m == 0 || n == 0) {
-            if (tid == 0) {
-                dist_out[idx] = max(m, n);
-                descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i), 0u, 0u};
-            }
-            continue;
-        }
-        const int32_t* txt = a.seqs + ((size_t)g * N + j) * a.stride;
-        uint16_t* loc = locs + idx * W.pitch;
-        for (int c = tid; c < n; c += kPrepThreads) {
-            const int32_t sym = __ldg(txt + c);
-            uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> hshift;
-            uint32_t v = kLocNone;
-            for (int probe = 0; probe < hslots; ++probe) {
-                const uint32_t o = s_owner[h];
-                if (o == 0u) break;
-                if (s_pat[o - 1u] == sym) {
-                    const uint32_t first = s_head[h] - 1u;
-                    v = s_next[first] == kChainEnd ? first : (kLocMulti | first);
-                    break;
-                }
-                h = (h + 1u) & (uint32_t)(hslots - 1);
-            }
-            loc[c] = (uint16_t)v;
-        }
-        if (tid == 0) {
+            dist_out[idx] = max(m, n);
+            descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i), 0u, 0u};
+        } else {
+            int tlog, R;
+            team_shape(m, tlog, R);
             const int bin = bin_of(n, tlog, R);
             descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i),
                                   (uint32_t)bin | 0x80000000u, 0u};
@@ -463,13 +496,10 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
 
     int hslots = 64;
     while (hslots < 2 * a.K) hslots <<= 1;
-    int hshift = 32;
-    while ((1 << (32 - hshift)) < hslots) --hshift;
-    const int prep_smem = W.pitch * 4 + hslots * 8 + W.pitch * 2;
+    const int prep_smem = W.pitch * 4 + hslots * 4 + W.pitch * 4;
 
-    if (ev) SR_CUDA_TRY(cudaEventRecord(ev[0], s));
     SR_CUDA_TRY(cudaMemsetAsync(ctl->hist, 0, sizeof(ctl->hist), s));
-    multi_prep_kernel<<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, hshift, dist);
+    multi_prep_kernel<<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist);
     SR_LAUNCH_CHECK("multi_prep_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[1], s));
     multi_scan_kernel<<<1, kNumBins, 0, s>>>(ctl);
