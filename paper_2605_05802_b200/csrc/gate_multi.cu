@@ -118,15 +118,22 @@ __device__ __forceinline__ int clamp_len(const int32_t* lens, size_t idx, int K,
 }
 
 // ------------------------------------------------------------------------ prep
+// A slot of the pattern's hash table: symbol in the high word, position of the
+// claiming occurrence + 1 in the low word (0 = empty slot), so that one 8-byte
+// shared-memory load answers "empty, this symbol, or another symbol".
+__device__ __forceinline__ unsigned long long make_slot(int32_t sym, uint32_t pos_plus_1) {
+    return ((unsigned long long)(uint32_t)sym << 32) | pos_plus_1;
+}
+
 // Position (or chain head) of `sym` in the pattern hashed in shared memory.
-__device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, const int32_t* s_pat,
-                                                   const uint32_t* s_owner, const uint32_t* s_next,
-                                                   int hslots, int hshift) {
+__device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, const unsigned long long* s_slot,
+                                                   const uint32_t* s_next, int hslots, int hshift) {
     uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> hshift;
     for (int probe = 0; probe < hslots; ++probe) {     // an empty slot always exists
-        const uint32_t o = s_owner[h];
+        const unsigned long long v = s_slot[h];
+        const uint32_t o = (uint32_t)v;
         if (o == 0u) break;
-        if (s_pat[o - 1u] == sym) {
+        if ((int32_t)(v >> 32) == sym) {
             const uint32_t first = o - 1u;
             return s_next[first] == kChainEnd ? first : (kLocMulti | first);
         }
@@ -135,12 +142,11 @@ __device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, const int32_t* s
     return kLocNone;
 }
 
-__global__ void __launch_bounds__(kPrepThreads)
+__global__ void __launch_bounds__(kPrepThreads, 8)
 multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int32_t* dist_out) {
     extern __shared__ __align__(16) unsigned char smem[];
-    int32_t* s_pat = reinterpret_cast<int32_t*>(smem);                       // [pitch]
-    uint32_t* s_owner = reinterpret_cast<uint32_t*>(s_pat + W.pitch);        // [hslots_max]
-    uint32_t* s_next = s_owner + hslots_max;                                 // [pitch]
+    unsigned long long* s_slot = reinterpret_cast<unsigned long long*>(smem);    // [hslots_max]
+    uint32_t* s_next = reinterpret_cast<uint32_t*>(s_slot + hslots_max);         // [pitch]
     __shared__ int s_txt[SR_MAX_N], s_len[SR_MAX_N], s_qstart[SR_MAX_N + 1], s_ntxt;
 
     const int N = a.N, K = a.K, P = pairs_of(N);
@@ -154,12 +160,9 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
     int hslots = 64;
     while (hslots < 2 * m) hslots <<= 1;
     const int hshift = __clz(hslots) + 1;             // 32 - log2(hslots)
-    const int32_t* pat = a.seqs + ((size_t)g * N + i) * a.stride;
-    for (int q = tid; 4 * q < m; q += kPrepThreads) {   // rows are 16-byte aligned, stride % 4 == 0
-        reinterpret_cast<int4*>(s_pat)[q] = __ldg(reinterpret_cast<const int4*>(pat) + q);
+    for (int q = tid; 4 * q < m; q += kPrepThreads)
         reinterpret_cast<uint4*>(s_next)[q] = make_uint4(kChainEnd, kChainEnd, kChainEnd, kChainEnd);
-    }
-    for (int h = tid; h < hslots; h += kPrepThreads) s_owner[h] = 0u;
+    for (int h = tid; h < hslots; h += kPrepThreads) s_slot[h] = 0ull;
     if (tid == 0) {                                   // the texts this pattern is paired with
         int cnt = 0, quads = 0;
         for (int j = 0; j < N; ++j) {
@@ -179,15 +182,17 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
     __syncthreads();
     // every position claims the slot of its symbol, or links itself behind the
     // position that claimed it (the claimant heads the symbol's occurrence chain)
+    const int32_t* pat = a.seqs + ((size_t)g * N + i) * a.stride;
     for (int p = tid; p < m; p += kPrepThreads) {
-        const int32_t sym = s_pat[p];
+        const int32_t sym = __ldg(pat + p);
         uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> hshift;
+        const unsigned long long mine = make_slot(sym, (uint32_t)p + 1u);
         for (int probe = 0; probe < hslots; ++probe) {
-            uint32_t o = s_owner[h];
-            if (o == 0u) o = atomicCAS(&s_owner[h], 0u, (uint32_t)p + 1u);
-            if (o == 0u) break;
-            if (s_pat[o - 1u] == sym) {
-                s_next[p] = atomicExch(&s_next[o - 1u], (uint32_t)p);
+            unsigned long long v = s_slot[h];
+            if ((uint32_t)v == 0u) v = atomicCAS(&s_slot[h], 0ull, mine);
+            if ((uint32_t)v == 0u) break;
+            if ((int32_t)(v >> 32) == sym) {
+                s_next[p] = atomicExch(&s_next[(uint32_t)v - 1u], (uint32_t)p);
                 break;
             }
             h = (h + 1u) & (uint32_t)(hslots - 1);
@@ -212,10 +217,10 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
         const int lo = min(i, j), hi = max(i, j);
         const size_t idx = (size_t)g * P + pair_index(lo, hi, N);
         const int4 sym = __ldg(reinterpret_cast<const int4*>(a.seqs + ((size_t)g * N + j) * a.stride) + q);
-        const uint32_t l0 = pattern_lookup(sym.x, s_pat, s_owner, s_next, hslots, hshift);
-        const uint32_t l1 = pattern_lookup(sym.y, s_pat, s_owner, s_next, hslots, hshift);
-        const uint32_t l2 = pattern_lookup(sym.z, s_pat, s_owner, s_next, hslots, hshift);
-        const uint32_t l3 = pattern_lookup(sym.w, s_pat, s_owner, s_next, hslots, hshift);
+        const uint32_t l0 = pattern_lookup(sym.x, s_slot, s_next, hslots, hshift);
+        const uint32_t l1 = pattern_lookup(sym.y, s_slot, s_next, hslots, hshift);
+        const uint32_t l2 = pattern_lookup(sym.z, s_slot, s_next, hslots, hshift);
+        const uint32_t l3 = pattern_lookup(sym.w, s_slot, s_next, hslots, hshift);
         reinterpret_cast<uint2*>(locs + idx * W.pitch)[q] = make_uint2(l0 | (l1 << 16), l2 | (l3 << 16));
     }
     if (tid < ntxt) {                                 // descriptors, bins, trivial pairs
@@ -496,8 +501,9 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
 
     int hslots = 64;
     while (hslots < 2 * a.K) hslots <<= 1;
-    const int prep_smem = W.pitch * 4 + hslots * 4 + W.pitch * 4;
+    const int prep_smem = hslots * 8 + W.pitch * 4;
 
+    if (ev) SR_CUDA_TRY(cudaEventRecord(ev[0], s));
     SR_CUDA_TRY(cudaMemsetAsync(ctl->hist, 0, sizeof(ctl->hist), s));
     multi_prep_kernel<<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist);
     SR_LAUNCH_CHECK("multi_prep_kernel");

@@ -1,0 +1,86 @@
+"""Run one of the synthetic workloads a few times through the C ABI and print its
+device time.  Handy for profiling a single kernel:
+
+    python -m paper_2605_05802_b200.run_case --case c3 --reps 3
+    ncu --set full --clock-control none -k regex:gate_single -c 1 \\
+        python -m paper_2605_05802_b200.run_case --case c3 --reps 3
+
+Cases: c1, c2, c3 (4096 groups x N=16), c3x16 (65536 groups), c4 (token level),
+c4s (256 groups), c5 (streaming, --groups to shrink), adv (advantages, 4M groups).
+"""
+from __future__ import annotations
+
+import argparse
+import statistics
+
+import torch
+
+import paper_2605_05802_b200 as sr
+from paper_2605_05802_b200 import workloads as W
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default="c3")
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--groups", type=int, default=0)
+    args = ap.parse_args()
+    dev = torch.device("cuda:0")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    times = []
+
+    def timed(fn):
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b) * 1e3)
+
+    if args.case in ("c1", "c2", "c3", "c3x16", "c4", "c4s"):
+        w = {"c1": lambda: W.tiny_gate(), "c2": lambda: W.agent_gate(K=15),
+             "c3": lambda: W.large_group_gate(n_groups=args.groups or 4096),
+             "c3x16": lambda: W.large_group_gate(n_groups=65536),
+             "c4": lambda: W.token_gate(n_groups=args.groups or 1024),
+             "c4s": lambda: W.token_gate(n_groups=256)}[args.case]()
+        G, N, stride = w.seqs.shape
+        seqs = torch.from_numpy(w.seqs).to(dev)
+        lens = torch.from_numpy(w.lens).to(dev)
+        ps = torch.empty(G, dtype=torch.int32, device=dev)
+        mean = torch.empty(G, dtype=torch.float64, device=dev)
+        stop = torch.empty(G, dtype=torch.uint8, device=dev)
+        wsb = sr.sr_gate_workspace_bytes(G, N, stride, w.K)
+        ws = torch.empty(wsb, dtype=torch.uint8, device=dev) if wsb else None
+        for _ in range(args.reps):
+            timed(lambda: sr.sr_gate(seqs, lens, w.K, w.threshold, w.norm_mode, pair_sum=ps, mean=mean,
+                                     stop=stop, workspace=ws))
+        print(f"{w.name}: {G} groups x N={N}, K={w.K}: median {statistics.median(times):.1f} us, "
+              f"{W.dp_cells(w.lens, w.K) / statistics.median(times) / 1e3:.0f} GCUPS, stopped {int(stop.sum())}")
+    elif args.case == "c5":
+        s = W.streaming_gate(n_groups=args.groups or 65536)
+        acts = torch.from_numpy(s.actions).to(dev)
+        state = torch.empty(sr.sr_incr_state_bytes(s.n_groups, s.N, s.steps), dtype=torch.uint8, device=dev)
+        mean = torch.empty(s.n_groups, dtype=torch.float64, device=dev)
+        stop = torch.empty(s.n_groups, dtype=torch.uint8, device=dev)
+        for _ in range(args.reps):
+            sr.sr_incr_init(state, s.n_groups, s.N, s.steps)
+            for t in range(s.steps):
+                timed(lambda: sr.sr_gate_step_incremental(state, acts[t], s.threshold, s.norm_mode,
+                                                          mean=mean, stop=stop))
+        print(f"{s.name}: {s.n_groups} groups, {s.steps} steps: median step {statistics.median(times):.1f} us, "
+              f"stopped at the end {int(stop.sum())}")
+    elif args.case == "adv":
+        G = args.groups or (64 * 65536)
+        r = torch.rand((G, 8), device=dev)
+        adv = torch.empty_like(r)
+        zv = torch.empty(G, dtype=torch.uint8, device=dev)
+        for _ in range(args.reps):
+            timed(lambda: sr.sr_grpo_advantage(r, None, 1e-6, adv=adv, zero_var=zv))
+        print(f"advantages: {G} groups x N=8: median {statistics.median(times):.1f} us")
+    else:
+        raise SystemExit(f"unknown case {args.case}")
+
+
+if __name__ == "__main__":
+    main()
