@@ -2,28 +2,55 @@
 // Section 3.2 of the paper: d_K at K <= T_max = 30).
 //
 // One CTA handles `gpb` consecutive groups.  Per group it
-//   1. stages the N prefixes once in shared memory (int4 loads),
+//   1. stages the N prefixes once in shared memory (int4 loads, rows of 32 words),
 //   2. renames the group's distinct IDs to dense local ids through a small
 //      open-addressing table in shared memory,
-//   3. builds the match masks Peq[i][id] (bit r set iff rollout i has symbol id at
-//      position r),
+//   3. builds, per rollout i, a byte map id -> a position of that symbol in rollout i
+//      and the match masks peq[i][position] (bit r set iff rollout i has the same
+//      symbol at r); the map costs one byte per (rollout, id) instead of one word,
+//      which is what lets several CTAs share an SM,
 //   4. runs one thread per pair through the bit-parallel column recurrence (one
 //      32-bit word of +1 / -1 vertical deltas per pair; the distance is read off as
 //      n + popc(Pv) - popc(Mv), so no per-column score is kept),
 //   5. adds the normalised terms in fp64 in pair order, thresholds, and writes out.
+// Index arithmetic uses shifts only (rows are 32 words), since integer division by a
+// run-time value costs more than a whole column of the recurrence.
 #include "common.cuh"
 
 namespace sr {
 namespace {
 
+// d / L for 0 <= d, L <= 32 (0 when L == 0), correctly rounded: the compiler's
+// constant evaluation of an IEEE division equals the device's __ddiv_rn.
+struct QuotientTable {
+    double v[33 * 33];
+    constexpr QuotientTable() : v() {
+        for (int d = 0; d <= 32; ++d)
+            for (int l = 0; l <= 32; ++l) v[d * 33 + l] = l > 0 ? (double)d / (double)l : 0.0;
+    }
+};
+__device__ const QuotientTable kQuot = QuotientTable();
+
+// Row pitch (16-bit elements) of the local-id rows: 17 words, so that pair threads
+// reading the same column of different rollouts hit different banks.
+constexpr int kGidPitch = 34;
+// Row pitch (words) of the per-rollout match masks: 32 masks indexed by a
+// representative position of the symbol, plus one all-zero mask for "absent".
+constexpr int kPeqPitch = 33;
+constexpr uint32_t kAbsent = 32;
+
 struct SingleLayout {
     int gpb;        // groups per CTA
-    int kpad;       // K rounded up to a multiple of 4 (<= 32)
     int hslots;     // hash slots per group (power of two)
     int hshift;     // 32 - log2(hslots)
-    int dmax;       // upper bound of distinct symbols per group (N * K)
-    // byte offsets into dynamic shared memory
-    int off_len, off_sym, off_gid, off_owner, off_cnt, off_peq, off_dist, off_term, off_pairs;
+    int mpitch;     // bytes per row of the id -> representative-position map (multiple of 4)
+    // Byte offsets into dynamic shared memory.  `off_build` holds the staged symbols and
+    // the hash table while the local ids are being assigned; once they are final the
+    // same bytes are reused for the map and the match masks.
+    int off_len, off_gid, off_cnt, off_dist, off_term, off_pairs, off_build;
+    int build_bytes;                       // per group
+    int sym_off, owner_off;                // within a group's build area (phase 1)
+    int map_off, peq_off;                  // within a group's build area (phase 2)
     int total;
 };
 
@@ -34,20 +61,24 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int g0 = blockIdx.x * L.gpb;
     const int ng = min(L.gpb, a.n_groups - g0);
+    const int rows = ng * N;                       // staged prefixes, 32 words each
+    const int per_group = N << 5;
 
-    int32_t* s_len = reinterpret_cast<int32_t*>(smem + L.off_len);          // [gpb][N]
-    int32_t* s_sym = reinterpret_cast<int32_t*>(smem + L.off_sym);          // [gpb][N][kpad]
-    uint16_t* s_gid = reinterpret_cast<uint16_t*>(smem + L.off_gid);        // [gpb][N][kpad]
-    uint32_t* s_owner = reinterpret_cast<uint32_t*>(smem + L.off_owner);    // [gpb][hslots]
+    int32_t* s_len = reinterpret_cast<int32_t*>(smem + L.off_len);          // [gpb*N]
+    uint16_t* s_gid = reinterpret_cast<uint16_t*>(smem + L.off_gid);        // [gpb*N][kGidPitch]
     int32_t* s_cnt = reinterpret_cast<int32_t*>(smem + L.off_cnt);          // [gpb]
-    uint32_t* s_peq = reinterpret_cast<uint32_t*>(smem + L.off_peq);        // [gpb][N][dmax]
     int32_t* s_dist = reinterpret_cast<int32_t*>(smem + L.off_dist);        // [gpb][P]
     double* s_term = reinterpret_cast<double*>(smem + L.off_term);          // [gpb][P]
     uint16_t* s_pairs = reinterpret_cast<uint16_t*>(smem + L.off_pairs);    // [P]  i | j << 8
+    unsigned char* s_build = smem + L.off_build;                            // [gpb][build_bytes]
+    auto sym_of = [&](int g) { return reinterpret_cast<int32_t*>(s_build + (size_t)g * L.build_bytes + L.sym_off); };
+    auto owner_of = [&](int g) { return reinterpret_cast<uint32_t*>(s_build + (size_t)g * L.build_bytes + L.owner_off); };
+    auto map_of = [&](int g) { return s_build + (size_t)g * L.build_bytes + L.map_off; };
+    auto peq_of = [&](int g) { return reinterpret_cast<uint32_t*>(s_build + (size_t)g * L.build_bytes + L.peq_off); };
 
-    // ---- lengths, pair table, table clears
+    // ---- lengths, pair table, hash-table clear
     bool neg = false;
-    for (int e = tid; e < ng * N; e += nthr) {
+    for (int e = tid; e < rows; e += nthr) {
         int len = a.lens ? a.lens[(size_t)g0 * N + e] : K;
         if (len < 0) { len = 0; neg = true; }
         s_len[e] = min(len, K);
@@ -58,62 +89,92 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
         pair_from_index(p, N, i, j);
         s_pairs[p] = (uint16_t)(i | (j << 8));
     }
-    for (int e = tid; e < ng * L.hslots; e += nthr) s_owner[e] = 0u;
+    for (int g = 0; g < ng; ++g) {
+        uint32_t* own = owner_of(g);
+        for (int e = tid; e < L.hslots; e += nthr) own[e] = 0u;
+    }
     if (tid < ng) s_cnt[tid] = 0;
 
-    // ---- stage the prefixes: one int4 per thread per trip, 16-byte aligned by contract
-    const int q4 = (K + 3) >> 2, pitch4 = L.kpad >> 2;   // q4 == 0 when K == 0: nothing to stage
-    for (int e = tid; e < ng * N * q4; e += nthr) {
-        const int row = e / q4, q = e - row * q4;
-        const int4 v = __ldg(reinterpret_cast<const int4*>(a.seqs + ((size_t)g0 * N + row) * a.stride) + q);
-        reinterpret_cast<int4*>(s_sym)[row * pitch4 + q] = v;
+    // ---- stage the prefixes: 8 lanes per row, one int4 each (16-byte aligned by contract)
+    const int q4 = (K + 3) >> 2;                   // 0 when K == 0: nothing to stage
+    for (int e = tid; e < rows * 8; e += nthr) {
+        const int row = e >> 3, q = e & 7;
+        if (q < q4) {
+            const int g = row / N, i = row - g * N;
+            const int4 v = __ldg(reinterpret_cast<const int4*>(a.seqs + ((size_t)g0 * N + row) * a.stride) + q);
+            reinterpret_cast<int4*>(sym_of(g))[i * 8 + q] = v;
+        }
     }
     __syncthreads();
 
     // ---- dense local ids: claim a slot per distinct symbol (slot identity = the
     // symbol of the claiming position), then number the claimed slots
-    const int per_group = N * L.kpad;
-    for (int e = tid; e < ng * per_group; e += nthr) {
-        const int g = e / per_group, rem = e - g * per_group;
-        const int i = rem / L.kpad, r = rem - i * L.kpad;
-        if (r >= s_len[g * N + i]) continue;
-        const int32_t sym = s_sym[e];
-        uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> L.hshift;
-        uint32_t* own = s_owner + g * L.hslots;
-        // the table has at least twice as many slots as symbols, so a free or matching
-        // slot is always found; the trip count is bounded all the same
-        for (int probe = 0; probe < L.hslots; ++probe) {
-            uint32_t o = own[h];
-            if (o == 0u) o = atomicCAS(&own[h], 0u, (uint32_t)rem + 1u);
-            if (o == 0u || s_sym[g * per_group + (int)o - 1] == sym) break;
-            h = (h + 1u) & (uint32_t)(L.hslots - 1);
-        }
-        s_gid[e] = (uint16_t)h;
-    }
-    __syncthreads();
-    for (int e = tid; e < ng * L.hslots; e += nthr) {
-        if (s_owner[e] != 0u) {
-            const int g = e / L.hslots;
-            s_owner[e] = (uint32_t)atomicAdd(&s_cnt[g], 1);
+    for (int g = 0; g < ng; ++g) {
+        uint32_t* own = owner_of(g);
+        const int32_t* sym_g = sym_of(g);
+        for (int e = tid; e < per_group; e += nthr) {
+            if ((e & 31) >= s_len[g * N + (e >> 5)]) continue;
+            const int32_t sym = sym_g[e];
+            uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> L.hshift;
+            // the table has at least twice as many slots as symbols, so a free or matching
+            // slot is always found; the trip count is bounded all the same
+            for (int probe = 0; probe < L.hslots; ++probe) {
+                uint32_t o = own[h];
+                if (o == 0u) o = atomicCAS(&own[h], 0u, (uint32_t)e + 1u);
+                if (o == 0u || sym_g[o - 1u] == sym) break;
+                h = (h + 1u) & (uint32_t)(L.hslots - 1);
+            }
+            s_gid[(g * N + (e >> 5)) * kGidPitch + (e & 31)] = (uint16_t)h;
         }
     }
     __syncthreads();
     for (int g = 0; g < ng; ++g) {
-        const int cnt = s_cnt[g];
-        uint32_t* peq = s_peq + (size_t)g * N * L.dmax;
-        for (int e = tid; e < N * cnt; e += nthr) {
-            const int i = e / cnt;
-            peq[i * L.dmax + (e - i * cnt)] = 0u;
+        uint32_t* own = owner_of(g);
+        for (int e = tid; e < L.hslots; e += nthr)
+            if (own[e] != 0u) own[e] = (uint32_t)atomicAdd(&s_cnt[g], 1);
+    }
+    __syncthreads();
+    for (int g = 0; g < ng; ++g) {
+        const uint32_t* own = owner_of(g);
+        for (int e = tid; e < per_group; e += nthr) {
+            if ((e & 31) >= s_len[g * N + (e >> 5)]) continue;
+            uint16_t* slot = s_gid + (g * N + (e >> 5)) * kGidPitch + (e & 31);
+            *slot = (uint16_t)own[*slot];
         }
     }
     __syncthreads();
-    for (int e = tid; e < ng * per_group; e += nthr) {
-        const int g = e / per_group, rem = e - g * per_group;
-        const int i = rem / L.kpad, r = rem - i * L.kpad;
-        if (r >= s_len[g * N + i]) continue;
-        const uint32_t gid = s_owner[g * L.hslots + s_gid[e]];
-        s_gid[e] = (uint16_t)gid;
-        atomicOr(&s_peq[((size_t)g * N + i) * L.dmax + gid], 1u << r);
+
+    // ---- the staged symbols and the hash table are dead; their bytes now hold, per
+    // rollout i, map[i][id] = a position of rollout i holding symbol id (kAbsent if none)
+    // and peq[i][pos] = bit mask of all positions of rollout i with the symbol found at pos
+    for (int g = 0; g < ng; ++g) {
+        uint32_t* map32 = reinterpret_cast<uint32_t*>(map_of(g));
+        const int words = (N * L.mpitch) >> 2;
+        for (int e = tid; e < words; e += nthr) map32[e] = kAbsent * 0x01010101u;
+        uint32_t* peq = peq_of(g);
+        for (int e = tid; e < N * kPeqPitch; e += nthr) peq[e] = 0u;
+    }
+    __syncthreads();
+    for (int g = 0; g < ng; ++g) {
+        volatile unsigned char* map = map_of(g);
+        for (int e = tid; e < per_group; e += nthr) {
+            const int i = e >> 5, r = e & 31;
+            if (r >= s_len[g * N + i]) continue;
+            // several positions with the same symbol store to the same byte; whichever store
+            // lands last names the representative, and any of them is a valid one
+            map[i * L.mpitch + s_gid[(g * N + i) * kGidPitch + r]] = (unsigned char)r;
+        }
+    }
+    __syncthreads();
+    for (int g = 0; g < ng; ++g) {
+        const unsigned char* map = map_of(g);
+        uint32_t* peq = peq_of(g);
+        for (int e = tid; e < per_group; e += nthr) {
+            const int i = e >> 5, r = e & 31;
+            if (r >= s_len[g * N + i]) continue;
+            const uint32_t rep = map[i * L.mpitch + s_gid[(g * N + i) * kGidPitch + r]];
+            atomicOr(&peq[i * kPeqPitch + rep], 1u << r);
+        }
     }
     __syncthreads();
 
@@ -125,11 +186,12 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
         const int mi = s_len[g * N + pi], mj = s_len[g * N + pj];
         int mp = mi, mt = mj;                       // pattern = the longer prefix (rows)
         if (mj > mi) { const int t = pi; pi = pj; pj = t; mp = mj; mt = mi; }
-        const uint32_t* peq = s_peq + ((size_t)g * N + pi) * L.dmax;
-        const uint16_t* txt = s_gid + (size_t)g * per_group + pj * L.kpad;
+        const unsigned char* map = map_of(g) + pi * L.mpitch;
+        const uint32_t* peq = peq_of(g) + pi * kPeqPitch;
+        const uint16_t* txt = s_gid + (g * N + pj) * kGidPitch;
         uint32_t Pv = 0xFFFFFFFFu, Mv = 0u;
         for (int c = 0; c < mt; ++c) {
-            const uint32_t Eq = peq[txt[c]];
+            const uint32_t Eq = peq[map[txt[c]]];
             const uint32_t Xv = Eq | Mv;
             const uint32_t Xh = (((Eq & Pv) + Pv) ^ Pv) | Eq;
             uint32_t Ph = Mv | ~(Xh | Pv);
@@ -142,19 +204,28 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
         const uint32_t msk = low_mask(mp);
         const int d = mt + __popc(Pv & msk) - __popc(Mv & msk);
         s_dist[tid] = d;
-        s_term[tid] = pair_term(d, mi, mj, a.norm_mode);
+        // one term of d_K (Section 3.2): distance / longer prefix, from the quotient table
+        s_term[tid] = a.norm_mode == SR_NORM_NONE ? (double)d : kQuot.v[d * 33 + mp];
         if (a.pair_dist) a.pair_dist[(size_t)g0 * P + tid] = d;
     }
     __syncthreads();
 
-    // ---- d_K: ordered fp64 sum, strict threshold (Eq. 2)
+    // ---- d_K: ordered fp64 sum, strict threshold (Eq. 2).  The loads are issued eight
+    // at a time ahead of the (necessarily sequential) additions.
     if (tid < ng) {
+        const double* term = s_term + tid * P;
+        const int32_t* dist = s_dist + tid * P;
         double s = 0.0;
-        int isum = 0;
-        for (int p = 0; p < P; ++p) {
-            s = __dadd_rn(s, s_term[tid * P + p]);
-            isum += s_dist[tid * P + p];
+        int isum = 0, p = 0;
+        for (; p + 8 <= P; p += 8) {
+            double t[8];
+            int d[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { t[u] = term[p + u]; d[u] = dist[p + u]; }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { s = __dadd_rn(s, t[u]); isum += d[u]; }
         }
+        for (; p < P; ++p) { s = __dadd_rn(s, term[p]); isum += dist[p]; }
         const double dk = __ddiv_rn(s, (double)P);
         if (a.pair_sum) a.pair_sum[g0 + tid] = isum;
         if (a.mean) a.mean[g0 + tid] = dk;
@@ -168,14 +239,23 @@ int launch_gate_single(const GateArgs& a, cudaStream_t s) {
     if (a.n_groups == 0) return SR_OK;
     const int N = a.N, P = pairs_of(N);
     SingleLayout L;
-    L.kpad = (a.K + 3) & ~3;
-    if (L.kpad == 0) L.kpad = 4;
-    L.dmax = N * a.K > 0 ? N * a.K : 1;
     int h = 32;
-    while (h < 2 * N * L.kpad) h <<= 1;
+    while (h < 2 * N * a.K) h <<= 1;
     L.hslots = h;
     L.hshift = 32;
     while ((1 << (32 - L.hshift)) < h) --L.hshift;
+    // map rows: one byte per distinct id (at most N*K), padded to an odd number of words
+    // so that consecutive rows start in different banks
+    int mwords = (N * a.K + 3) >> 2;
+    if ((mwords & 1) == 0) ++mwords;
+    L.mpitch = mwords * 4;
+    L.sym_off = 0;
+    L.owner_off = N * 32 * 4;
+    L.map_off = 0;
+    L.peq_off = (N * L.mpitch + 15) & ~15;
+    const int phase1 = L.owner_off + L.hslots * 4;
+    const int phase2 = L.peq_off + N * kPeqPitch * 4;
+    L.build_bytes = ((phase1 > phase2 ? phase1 : phase2) + 15) & ~15;
     int gpb = 256 / P;
     if (gpb < 1) gpb = 1;
     if (gpb > 32) gpb = 32;
@@ -187,17 +267,14 @@ int launch_gate_single(const GateArgs& a, cudaStream_t s) {
         int off = 0;
         auto take = [&](int bytes) { int o = off; off = (off + bytes + 15) & ~15; return o; };
         L.off_len = take(gpb * N * 4);
-        L.off_sym = take(gpb * N * L.kpad * 4);
-        L.off_gid = take(gpb * N * L.kpad * 2);
-        L.off_owner = take(gpb * L.hslots * 4);
+        L.off_gid = take(gpb * N * kGidPitch * 2);
         L.off_cnt = take(gpb * 4);
-        L.off_peq = take(gpb * N * L.dmax * 4);
         L.off_dist = take(gpb * P * 4);
         L.off_term = take(gpb * P * 8);
         L.off_pairs = take(P * 2);
+        L.off_build = take(gpb * L.build_bytes);
         L.total = off;
-        // keep at least two CTAs per SM when the group count allows it
-        if (L.total <= max_smem / 2 || gpb == 1) break;
+        if (L.total <= max_smem / 4 || gpb == 1) break;   // leave room for several CTAs per SM
         --gpb;
     }
     if (L.total > max_smem) return SR_ERR_BAD_N;
