@@ -15,7 +15,10 @@
 // State buffer layout (position independent, byte-copyable):
 //   [0, 256)        header: magic, n_groups, N, max_steps
 //   lens   int32 [n_groups][N]
-//   hist   int32 [n_groups][N][32]        actions emitted so far
+//   hist   int32 [n_groups][8][N][4]      actions emitted so far: action r of rollout i
+//                                         sits at [r / 4][i][r % 4], so that the first
+//                                         quads of all rollouts of a group (what a step
+//                                         reads) are contiguous
 //   pairs  uint4 [n_groups][P]            (VP, VN, HP, HN)
 // every section starts on a 256-byte boundary.
 #include "common.cuh"
@@ -97,88 +100,127 @@ struct IncrArgs {
     uint8_t* stop;
     int32_t* status;
     int gpb;
-    int off_len, off_new, off_hist, off_dist, off_term, off_pairs;   // shared-memory offsets
+    int off_dist, off_term;                                // shared-memory offsets
 };
 
-__global__ void __launch_bounds__(1024)
+// d / L for 0 <= d, L <= 32 (0 when L == 0), correctly rounded: the compiler's
+// constant evaluation of an IEEE division equals the device's __ddiv_rn.
+struct QuotientTable {
+    double v[33 * 33];
+    constexpr QuotientTable() : v() {
+        for (int d = 0; d <= 32; ++d)
+            for (int l = 0; l <= 32; ++l) v[d * 33 + l] = l > 0 ? (double)d / (double)l : 0.0;
+    }
+};
+__device__ const QuotientTable kQuot = QuotientTable();
+
+// Bit r set iff action r of rollout `i` equals sym, for r < len.  `quads` points at the
+// group's stored actions ([8][N] int4); four actions per load; positions >= len are
+// masked off, so whatever those words hold does not matter.
+__device__ __forceinline__ uint32_t match_mask(const int4* quads, int N, int i, int len, int32_t sym) {
+    uint32_t eq = 0u;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        if (4 * q < len) {
+            const int4 v = quads[q * N + i];
+            eq |= (v.x == sym ? 1u : 0u) << (4 * q);
+            eq |= (v.y == sym ? 2u : 0u) << (4 * q);
+            eq |= (v.z == sym ? 4u : 0u) << (4 * q);
+            eq |= (v.w == sym ? 8u : 0u) << (4 * q);
+        }
+    }
+    return eq & low_mask(len);
+}
+
+// (i, j) of pair p for every group size: filled in at compile time.
+struct PairTable {
+    uint16_t v[SR_MAX_N + 1][SR_MAX_N * (SR_MAX_N - 1) / 2];
+    constexpr PairTable() : v() {
+        for (int n = 2; n <= SR_MAX_N; ++n) {
+            int p = 0;
+            for (int i = 0; i < n; ++i)
+                for (int j = i + 1; j < n; ++j) v[n][p++] = (uint16_t)(i | (j << 8));
+        }
+    }
+};
+__device__ const PairTable kPairs = PairTable();
+
+// One thread per pair, `gpb` groups per CTA.  Everything a pair needs (its state, the
+// two lengths, the two new actions, the header) is requested in one round of
+// independent loads; the stored actions follow in a second round; only then does the
+// CTA synchronise, once before the appends and once before the per-group sums.
+__global__ void __launch_bounds__(512, 4)
 incr_step_kernel(IncrArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int N = a.N, P = pairs_of(N);
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int g0 = blockIdx.x * a.gpb;
     const int ng = min(a.gpb, a.n_groups - g0);
-    const uint32_t* hdr = reinterpret_cast<const uint32_t*>(a.state);
-    if (hdr[0] != kMagic || hdr[1] != (uint32_t)a.n_groups || hdr[2] != (uint32_t)N) {
-        if (tid == 0 && a.status) atomicOr(a.status, SR_STATUS_BAD_STATE);
-        return;
-    }
-    const int max_steps = (int)hdr[3];
-
-    int32_t* s_len = reinterpret_cast<int32_t*>(smem + a.off_len);      // [gpb][N] old lengths
-    int32_t* s_new = reinterpret_cast<int32_t*>(smem + a.off_new);      // [gpb][N] new action
-    int32_t* s_hist = reinterpret_cast<int32_t*>(smem + a.off_hist);    // [gpb][N][33]
     int32_t* s_dist = reinterpret_cast<int32_t*>(smem + a.off_dist);    // [gpb][P]
     double* s_term = reinterpret_cast<double*>(smem + a.off_term);      // [gpb][P]
-    uint16_t* s_pairs = reinterpret_cast<uint16_t*>(smem + a.off_pairs);
 
+    const uint4 hdr = *reinterpret_cast<const uint4*>(a.state);         // magic, n_groups, N, max_steps
     int32_t* g_len = reinterpret_cast<int32_t*>(a.state + a.L.off_lens) + (size_t)g0 * N;
     int32_t* g_hist = reinterpret_cast<int32_t*>(a.state + a.L.off_hist) + (size_t)g0 * N * kHistPitch;
     uint4* g_pairs = reinterpret_cast<uint4*>(a.state + a.L.off_pairs) + (size_t)g0 * P;
+    const int32_t* g_new = a.new_actions + (size_t)g0 * N;
 
-    bool overflow = false;
-    for (int e = tid; e < ng * N; e += nthr) {
-        const int len = g_len[e];
-        int32_t act = __ldg(a.new_actions + (size_t)g0 * N + e);
-        if (act != SR_NO_ACTION && len >= max_steps) { act = SR_NO_ACTION; overflow = true; }
-        s_len[e] = len;
-        s_new[e] = act;
-    }
-    if (overflow && a.status) atomicOr(a.status, SR_STATUS_STEP_OVERFLOW);
-    for (int p = tid; p < P; p += nthr) {
-        int i, j;
-        pair_from_index(p, N, i, j);
-        s_pairs[p] = (uint16_t)(i | (j << 8));
-    }
-    __syncthreads();
-    // history so far -> shared memory (rows padded to 33 words: pair threads of one
-    // warp read different rows at the same position)
-    for (int e = tid; e < ng * N * kHistPitch; e += nthr) {
-        const int row = e >> 5, r = e & 31;
-        if (r < s_len[row]) s_hist[row * 33 + r] = g_hist[e];
-    }
-    __syncthreads();
-    // append this step's actions to the stored history and lengths
-    for (int e = tid; e < ng * N; e += nthr) {
-        if (s_new[e] != SR_NO_ACTION) {
-            g_hist[e * kHistPitch + s_len[e]] = s_new[e];
-            g_len[e] = s_len[e] + 1;
-        }
-    }
-
-    if (tid < ng * P) {
+    const bool is_pair = tid < ng * P;
+    uint4 st = make_uint4(0u, 0u, 0u, 0u);
+    int gi = 0, gj = 0, m = 0, n = 0, grp = 0;
+    int32_t x = SR_NO_ACTION, y = SR_NO_ACTION;
+    if (is_pair) {
         const int g = tid / P, p = tid - g * P;
-        const int pr = s_pairs[p];
-        const int i = pr & 0xFF, j = pr >> 8;
-        const int m = s_len[g * N + i], n = s_len[g * N + j];
-        const int32_t x = s_new[g * N + i], y = s_new[g * N + j];
+        const int pr = kPairs.v[N][p];
+        grp = g;
+        gi = g * N + (pr & 0xFF);
+        gj = g * N + (pr >> 8);
+        st = g_pairs[tid];
+        m = g_len[gi];
+        n = g_len[gj];
+        x = __ldg(g_new + gi);
+        y = __ldg(g_new + gj);
+    }
+    // appenders: thread e < ng*N owns rollout e of this CTA
+    const bool is_roll = tid < ng * N;
+    int my_len = 0;
+    int32_t my_act = SR_NO_ACTION;
+    if (is_roll) { my_len = g_len[tid]; my_act = __ldg(g_new + tid); }
+
+    const bool bad = hdr.x != kMagic || hdr.y != (uint32_t)a.n_groups || hdr.z != (uint32_t)N;
+    if (bad) {                                     // uniform over the grid: nothing is touched
+        if (tid == 0 && a.status) atomicOr(a.status, SR_STATUS_BAD_STATE);
+        return;
+    }
+    const int max_steps = (int)hdr.w;
+    if (x != SR_NO_ACTION && m >= max_steps) x = SR_NO_ACTION;     // rollout already full: ignored
+    if (y != SR_NO_ACTION && n >= max_steps) y = SR_NO_ACTION;
+    if (is_roll && my_act != SR_NO_ACTION && my_len >= max_steps) {
+        my_act = SR_NO_ACTION;
+        if (a.status) atomicOr(a.status, SR_STATUS_STEP_OVERFLOW);
+    }
+
+    int hout = 1, vout = 1;
+    uint32_t VP2 = st.x, VN2 = st.y, HP2 = st.z, HN2 = st.w;
+    if (is_pair) {
+        // the stored actions are read straight from the state (the pairs of a group share
+        // N rows, so all but the first touch of a row hit L1)
+        const int4* quads = reinterpret_cast<const int4*>(g_hist) + (size_t)grp * 8 * N;
+        if (y != SR_NO_ACTION && m > 0)
+            hout = column_step(match_mask(quads, N, gi - grp * N, m, y), VP2, VN2, m);
+        if (x != SR_NO_ACTION && n > 0)
+            vout = column_step(match_mask(quads, N, gj - grp * N, n, x), HP2, HN2, n);
+    }
+    __syncthreads();       // every read of the stored actions precedes this step's appends
+    if (is_roll && my_act != SR_NO_ACTION) {
+        const int g = tid / N, i = tid - g * N;
+        g_hist[(((size_t)g * 8 + (my_len >> 2)) * N + i) * 4 + (my_len & 3)] = my_act;
+        g_len[tid] = my_len + 1;
+    }
+    if (is_pair) {
         const bool ai = x != SR_NO_ACTION, aj = y != SR_NO_ACTION;
-        uint4 st = g_pairs[tid];
         uint32_t VP = st.x, VN = st.y, HP = st.z, HN = st.w;
         const int c = n + __popc(VP) - __popc(VN);
-        int hout = 1, vout = 1;
-        uint32_t VP2 = VP, VN2 = VN, HP2 = HP, HN2 = HN;
-        if (aj && m > 0) {
-            const int32_t* hi = s_hist + (g * N + i) * 33;
-            uint32_t Eq = 0u;
-            for (int r = 0; r < m; ++r) Eq |= (hi[r] == y ? 1u : 0u) << r;
-            hout = column_step(Eq, VP2, VN2, m);
-        }
-        if (ai && n > 0) {
-            const int32_t* hj = s_hist + (g * N + j) * 33;
-            uint32_t Eq = 0u;
-            for (int r = 0; r < n; ++r) Eq |= (hj[r] == x ? 1u : 0u) << r;
-            vout = column_step(Eq, HP2, HN2, n);
-        }
         int d = c, mi = m, mj = n;
         if (ai && aj) {
             const int left = c + vout, up = c + hout;
@@ -204,17 +246,24 @@ incr_step_kernel(IncrArgs a) {
         }
         if (ai || aj) g_pairs[tid] = make_uint4(VP, VN, HP, HN);
         s_dist[tid] = d;
-        s_term[tid] = pair_term(d, mi, mj, a.norm_mode);
+        s_term[tid] = a.norm_mode == SR_NORM_NONE ? (double)d : kQuot.v[d * 33 + max(mi, mj)];
         if (a.pair_dist) a.pair_dist[(size_t)g0 * P + tid] = d;
     }
     __syncthreads();
     if (tid < ng) {
+        const double* term = s_term + tid * P;
+        const int32_t* dist = s_dist + tid * P;
         double s = 0.0;
-        int isum = 0;
-        for (int p = 0; p < P; ++p) {
-            s = __dadd_rn(s, s_term[tid * P + p]);
-            isum += s_dist[tid * P + p];
+        int isum = 0, p = 0;
+        for (; p + 8 <= P; p += 8) {               // loads ahead of the sequential additions
+            double t[8];
+            int dd[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { t[u] = term[p + u]; dd[u] = dist[p + u]; }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { s = __dadd_rn(s, t[u]); isum += dd[u]; }
         }
+        for (; p < P; ++p) { s = __dadd_rn(s, term[p]); isum += dist[p]; }
         const double dk = __ddiv_rn(s, (double)P);
         if (a.pair_sum) a.pair_sum[g0 + tid] = isum;
         if (a.mean) a.mean[g0 + tid] = dk;
@@ -260,19 +309,15 @@ int launch_incr_step(void* state, size_t bytes, const int32_t* new_actions, int3
     int gpb = 256 / P;
     if (gpb < 1) gpb = 1;
     if (gpb > 32) gpb = 32;
+    while (gpb > 1 && gpb * N > 256) --gpb;      // one appending thread per rollout
     a.gpb = gpb;
     int off = 0;
     auto take = [&](int b) { int o = off; off = (off + b + 15) & ~15; return o; };
-    a.off_len = take(gpb * N * 4);
-    a.off_new = take(gpb * N * 4);
-    a.off_hist = take(gpb * N * 33 * 4);
     a.off_dist = take(gpb * P * 4);
     a.off_term = take(gpb * P * 8);
-    a.off_pairs = take(P * 2);
     int threads = (gpb * P + 31) & ~31;
+    if (threads < gpb * N) threads = (gpb * N + 31) & ~31;
     if (threads < 64) threads = 64;
-    if (off > 48 * 1024)
-        SR_CUDA_TRY(cudaFuncSetAttribute(incr_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, off));
     const int blocks = (n_groups + gpb - 1) / gpb;
     incr_step_kernel<<<blocks, threads, off, s>>>(a);
     SR_LAUNCH_CHECK("incr_step_kernel");

@@ -27,10 +27,14 @@ def main():
     args = ap.parse_args()
     dev = torch.device("cuda:0")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    sweep = torch.zeros(64 << 20, dtype=torch.float32, device=dev)
     times = []
 
     def timed(fn):
+        # flush L2: write 256 MiB, then read another 256 MiB so that the dirty lines of
+        # the write are already back in DRAM when the timed launch starts
         flush.fill_(1)
+        sweep.sum()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         fn()
@@ -68,8 +72,10 @@ def main():
             for t in range(s.steps):
                 timed(lambda: sr.sr_gate_step_incremental(state, acts[t], s.threshold, s.norm_mode,
                                                           mean=mean, stop=stop))
+        per_step = [statistics.median(times[t::s.steps]) for t in range(s.steps)]
         print(f"{s.name}: {s.n_groups} groups, {s.steps} steps: median step {statistics.median(times):.1f} us, "
               f"stopped at the end {int(stop.sum())}")
+        print("  per step (us): " + " ".join(f"{v:.0f}" for v in per_step))
     elif args.case == "adv":
         G = args.groups or (64 * 65536)
         r = torch.rand((G, 8), device=dev)
