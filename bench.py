@@ -199,14 +199,14 @@ def main():
         flush.fill_(tag & 0xFF)
         sweep.sum()
 
-    def timed(fn, reps, warm=3, flush_l2=True):
+    def timed(fn, reps, warm=3, do_flush=True):
         """Per-launch device times (ms) of fn, L2 flushed before every launch."""
         for _ in range(warm):
             fn()
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
         torch.cuda.synchronize()
         for i, (a, b) in enumerate(evs):
-            if flush_l2:
+            if do_flush:
                 flush_l2(i)
             a.record()
             fn()
@@ -334,7 +334,7 @@ def main():
         sink = torch.empty(sms * 8 * 256, dtype=torch.int32, device=dev)
         probe = {}
         for name, var in (("logic", sr.SR_PROBE_LOGIC), ("add", sr.SR_PROBE_ADD), ("mix8l2a", sr.SR_PROBE_MIX)):
-            ms = min(timed(lambda: sr.sr_probe_int32(var, 2000, sms * 8, 256, sink), 5, flush_l2=False))
+            ms = min(timed(lambda: sr.sr_probe_int32(var, 2000, sms * 8, 256, sink), 5, do_flush=False))
             probe[name] = sr.sr_probe_int32_ops(2000, sms * 8, 256) / (ms * 1e-3) / 1e9
         extras["int32_probe_gops"] = probe
         # the recurrence is 8 logic : 2 add; logic issues on the int32 ALU only, adds can also
