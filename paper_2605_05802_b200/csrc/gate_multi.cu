@@ -520,9 +520,10 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     SR_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     // persistent grid: a multiple of the SM count; warps pull tasks until none is left
     long long want = (n_pairs_ll + kDpWarpsPerCta - 1) / kDpWarpsPerCta;
-    // 4 CTAs of 4 warps per SM: enough warps to keep the integer pipe busy, few enough
-    // that most tasks are pulled dynamically, longest first
-    long long cap = (long long)sms * 4;
+    // 3 CTAs of 4 warps per SM (3 warps per scheduler): enough to keep the integer pipe
+    // busy, few enough that most tasks are pulled dynamically, longest first (measured
+    // best among 2..6 warps per scheduler)
+    long long cap = (long long)sms * 3;
     int blocks = (int)(want < cap ? want : cap);
     if (blocks < 1) blocks = 1;
     multi_dp_kernel<<<blocks, kDpWarpsPerCta * 32, 0, s>>>(ws, W, dist, 2u);
