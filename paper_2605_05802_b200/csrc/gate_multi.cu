@@ -156,9 +156,11 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
     if (i >= M) return;                               // the last rollout of an even group is never a pattern
     bool neg = false;
     const int m = clamp_len(a.lens, (size_t)g * N + i, K, neg);
-    // the table holds at least twice as many slots as the pattern has symbols
+    // the table holds at least four times as many slots as the pattern has symbols:
+    // short probe sequences matter more than shared memory here (lanes wait for the
+    // longest probe of their warp)
     int hslots = 64;
-    while (hslots < 2 * m) hslots <<= 1;
+    while (hslots < 4 * m) hslots <<= 1;
     const int hshift = __clz(hslots) + 1;             // 32 - log2(hslots)
     for (int q = tid; 4 * q < m; q += kPrepThreads)
         reinterpret_cast<uint4*>(s_next)[q] = make_uint4(kChainEnd, kChainEnd, kChainEnd, kChainEnd);
@@ -500,7 +502,7 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     Ctl* ctl = reinterpret_cast<Ctl*>(ws + W.off_ctl);
 
     int hslots = 64;
-    while (hslots < 2 * a.K) hslots <<= 1;
+    while (hslots < 4 * a.K) hslots <<= 1;
     const int prep_smem = hslots * 8 + W.pitch * 4;
 
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[0], s));
