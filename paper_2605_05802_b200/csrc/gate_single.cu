@@ -49,7 +49,7 @@ struct SingleLayout {
     // same bytes are reused for the map and the match masks.
     int off_len, off_gid, off_cnt, off_dist, off_term, off_pairs, off_build;
     int build_bytes;                       // per group
-    int sym_off, owner_off;                // within a group's build area (phase 1)
+    int sym_off, owner_off, sgid_off;      // within a group's build area (phase 1)
     int map_off, peq_off;                  // within a group's build area (phase 2)
     int total;
 };
@@ -73,6 +73,7 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
     unsigned char* s_build = smem + L.off_build;                            // [gpb][build_bytes]
     auto sym_of = [&](int g) { return reinterpret_cast<int32_t*>(s_build + (size_t)g * L.build_bytes + L.sym_off); };
     auto owner_of = [&](int g) { return reinterpret_cast<uint32_t*>(s_build + (size_t)g * L.build_bytes + L.owner_off); };
+    auto sgid_of = [&](int g) { return reinterpret_cast<uint16_t*>(s_build + (size_t)g * L.build_bytes + L.sgid_off); };
     auto map_of = [&](int g) { return s_build + (size_t)g * L.build_bytes + L.map_off; };
     auto peq_of = [&](int g) { return reinterpret_cast<uint32_t*>(s_build + (size_t)g * L.build_bytes + L.peq_off); };
 
@@ -108,9 +109,10 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
     __syncthreads();
 
     // ---- dense local ids: claim a slot per distinct symbol (slot identity = the
-    // symbol of the claiming position), then number the claimed slots
+    // symbol of the claiming position); the claimant draws the group's next free id
     for (int g = 0; g < ng; ++g) {
         uint32_t* own = owner_of(g);
+        uint16_t* sgid = sgid_of(g);
         const int32_t* sym_g = sym_of(g);
         for (int e = tid; e < per_group; e += nthr) {
             if ((e & 31) >= s_len[g * N + (e >> 5)]) continue;
@@ -121,7 +123,8 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
             for (int probe = 0; probe < L.hslots; ++probe) {
                 uint32_t o = own[h];
                 if (o == 0u) o = atomicCAS(&own[h], 0u, (uint32_t)e + 1u);
-                if (o == 0u || sym_g[o - 1u] == sym) break;
+                if (o == 0u) { sgid[h] = (uint16_t)atomicAdd(&s_cnt[g], 1); break; }
+                if (sym_g[o - 1u] == sym) break;
                 h = (h + 1u) & (uint32_t)(L.hslots - 1);
             }
             s_gid[(g * N + (e >> 5)) * kGidPitch + (e & 31)] = (uint16_t)h;
@@ -129,17 +132,11 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
     }
     __syncthreads();
     for (int g = 0; g < ng; ++g) {
-        uint32_t* own = owner_of(g);
-        for (int e = tid; e < L.hslots; e += nthr)
-            if (own[e] != 0u) own[e] = (uint32_t)atomicAdd(&s_cnt[g], 1);
-    }
-    __syncthreads();
-    for (int g = 0; g < ng; ++g) {
-        const uint32_t* own = owner_of(g);
+        const uint16_t* sgid = sgid_of(g);
         for (int e = tid; e < per_group; e += nthr) {
             if ((e & 31) >= s_len[g * N + (e >> 5)]) continue;
             uint16_t* slot = s_gid + (g * N + (e >> 5)) * kGidPitch + (e & 31);
-            *slot = (uint16_t)own[*slot];
+            *slot = sgid[*slot];
         }
     }
     __syncthreads();
@@ -147,12 +144,12 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
     // ---- the staged symbols and the hash table are dead; their bytes now hold, per
     // rollout i, map[i][id] = a position of rollout i holding symbol id (kAbsent if none)
     // and peq[i][pos] = bit mask of all positions of rollout i with the symbol found at pos
-    for (int g = 0; g < ng; ++g) {
-        uint32_t* map32 = reinterpret_cast<uint32_t*>(map_of(g));
-        const int words = (N * L.mpitch) >> 2;
-        for (int e = tid; e < words; e += nthr) map32[e] = kAbsent * 0x01010101u;
-        uint32_t* peq = peq_of(g);
-        for (int e = tid; e < N * kPeqPitch; e += nthr) peq[e] = 0u;
+    for (int g = 0; g < ng; ++g) {                 // 16-byte stores: map = "absent", masks = 0
+        uint4* init = reinterpret_cast<uint4*>(map_of(g));
+        const int map_q = L.peq_off >> 4, all_q = (L.peq_off + ((N * kPeqPitch * 4 + 15) & ~15)) >> 4;
+        const uint32_t absent4 = kAbsent * 0x01010101u;
+        for (int e = tid; e < all_q; e += nthr)
+            init[e] = e < map_q ? make_uint4(absent4, absent4, absent4, absent4) : make_uint4(0u, 0u, 0u, 0u);
     }
     __syncthreads();
     for (int g = 0; g < ng; ++g) {
@@ -253,8 +250,9 @@ int launch_gate_single(const GateArgs& a, cudaStream_t s) {
     L.owner_off = N * 32 * 4;
     L.map_off = 0;
     L.peq_off = (N * L.mpitch + 15) & ~15;
-    const int phase1 = L.owner_off + L.hslots * 4;
-    const int phase2 = L.peq_off + N * kPeqPitch * 4;
+    L.sgid_off = L.owner_off + L.hslots * 4;
+    const int phase1 = L.sgid_off + L.hslots * 2;
+    const int phase2 = L.peq_off + ((N * kPeqPitch * 4 + 15) & ~15);
     L.build_bytes = ((phase1 > phase2 ? phase1 : phase2) + 15) & ~15;
     int gpb = 256 / P;
     if (gpb < 1) gpb = 1;
