@@ -182,6 +182,24 @@ int sr_gate_step_incremental(void* state, size_t state_bytes, const int32_t* new
                              int32_t* status, void* stream);
 
 /*
+ * sr_gate_or_rule -- termination fraction tau_K (Appendix B, "termination_fraction")
+ * and the two-clause gate of the OR-rule extension (Eq. 3):
+ *     stop[g] = (mean[g] < threshold) || (tau[g] >= tau_high),
+ * tau[g] = (finished rollouts of group g) / N in fp64.  A rollout counts as finished
+ * by step K when its `done` byte is non-zero or, when done == NULL, when it has emitted
+ * fewer than K actions (lens[g][i] < K).  tau_high > 1 reduces the rule to Eq. 2.
+ *
+ *   mean  in  [n_groups] fp64, d_K as written by sr_gate
+ *   lens  in  [n_groups][N] int32; required when done == NULL
+ *   done  in  [n_groups][N] uint8 or NULL
+ *   tau   out [n_groups] fp64; may be NULL
+ *   stop  out [n_groups] uint8; required
+ */
+int sr_gate_or_rule(const double* mean, const int32_t* lens, const uint8_t* done, int32_t n_groups,
+                    int32_t N, int32_t K, double threshold, double tau_high, double* tau,
+                    uint8_t* stop, void* stream);
+
+/*
  * sr_grpo_advantage -- Eq. 1: A_i = (r_i - mean_r) / (sigma_r + eps) with the
  * population standard deviation (1/N), accumulated in fp64 and rounded once to
  * fp32.  zero_var[g] = 1 iff all N rewards of the group compare equal (Section
@@ -196,6 +214,33 @@ int sr_gate_step_incremental(void* state, size_t state_bytes, const int32_t* new
  */
 int sr_grpo_advantage(const float* rewards, const uint8_t* drop_mask, int32_t n_groups,
                       int32_t N, float eps, float* adv, uint8_t* zero_var, void* stream);
+
+/*
+ * sr_batch_stats -- batch reductions behind two of the paper's figures: the share of
+ * zero-advantage trajectories that dilutes the batch-mean loss (Section 4.5: about 40 %
+ * without the gate, 28 % with it) and the advantage norm kept after cutting,
+ * ||A_kept||_2 / ||A_full||_2 (Section 3.4: 96.7 % at the chosen threshold).
+ *
+ *   adv     in  [n_groups][N] fp32 advantages computed WITHOUT a drop mask
+ *   stop    in  [n_groups] uint8 gate decisions, or NULL (every group kept)
+ *   counts  out 3 int64: [0] advantages equal to zero over all groups,
+ *                        [1] the same over kept groups (stop == 0), [2] kept groups
+ *   sumsq   out 2 fp64:  [0] sum of squared advantages over all groups, [1] over kept
+ *
+ * The fp64 sums are accumulated in parallel (thread, block, then atomics), so they are
+ * reproducible to about 1e-12 relative, not bit for bit; the counts are exact.
+ */
+int sr_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int32_t N,
+                   int64_t* counts, double* sumsq, void* stream);
+
+/* Host-only, pure.  Step-token saving of cutting `cut` of `n_groups` groups at step K of
+ * a horizon of T_max steps: cut * (T_max - K) / (n_groups * T_max) (caption of Table 1). */
+double sr_savings_fraction(int64_t cut, int64_t n_groups, int32_t T_max, int32_t K);
+
+/* Host-only, pure.  Gradient-norm gain predicted by the dilution argument when the
+ * zero-advantage fraction goes from `before` to `after`: (1 - after) / (1 - before)
+ * (Section 4.5: 0.72 / 0.60, about 1.20). */
+double sr_dilution_gain(double zero_frac_before, double zero_frac_after);
 
 #ifdef __cplusplus
 }

@@ -55,6 +55,17 @@ def _load():
         lib.sro_advantage.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
                                       ctypes.c_int32, ctypes.c_float, ctypes.c_void_p,
                                       ctypes.c_void_p]
+        lib.sro_or_rule.restype = None
+        lib.sro_or_rule.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
+                                    ctypes.c_int32, ctypes.c_int32, ctypes.c_double, ctypes.c_double,
+                                    ctypes.c_void_p, ctypes.c_void_p]
+        lib.sro_batch_stats.restype = None
+        lib.sro_batch_stats.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                        ctypes.c_void_p, ctypes.c_void_p]
+        lib.sro_savings_fraction.restype = ctypes.c_double
+        lib.sro_savings_fraction.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32]
+        lib.sro_dilution_gain.restype = ctypes.c_double
+        lib.sro_dilution_gain.argtypes = [ctypes.c_double, ctypes.c_double]
         lib.sro_max_threads.restype = ctypes.c_int32
         _lib = lib
     return _lib
@@ -112,6 +123,51 @@ def advantage(rewards: np.ndarray, drop_mask: Optional[np.ndarray] = None, eps: 
     _load().sro_advantage(rewards.ctypes.data, dp, G, N, float(np.float32(eps)), adv.ctypes.data,
                           zv.ctypes.data)
     return adv, zv
+
+
+def or_rule(mean: np.ndarray, lens: Optional[np.ndarray], done: Optional[np.ndarray], K: int,
+            threshold: float, tau_high: float):
+    """tau_K (fraction of finished rollouts) and the OR-rule mask of Eq. 3.
+    Returns (tau float64 [G], stop uint8 [G])."""
+    mean = np.ascontiguousarray(mean, dtype=np.float64)
+    G = mean.shape[0]
+    lp = dp = None
+    if done is not None:
+        done = np.ascontiguousarray(done, dtype=np.uint8)
+        N = done.shape[1]
+        dp = done.ctypes.data
+    if lens is not None:
+        lens = np.ascontiguousarray(lens, dtype=np.int32)
+        N = lens.shape[1]
+        lp = lens.ctypes.data
+    tau = np.zeros(G, dtype=np.float64)
+    stop = np.zeros(G, dtype=np.uint8)
+    _load().sro_or_rule(mean.ctypes.data, lp, dp, G, N, int(K), float(threshold), float(tau_high),
+                        tau.ctypes.data, stop.ctypes.data)
+    return tau, stop
+
+
+def batch_stats(adv: np.ndarray, stop: Optional[np.ndarray]):
+    """(counts int64 [3], sumsq float64 [2]): zero advantages over all / kept groups,
+    kept groups; squared advantage norm over all / kept groups."""
+    adv = np.ascontiguousarray(adv, dtype=np.float32)
+    G, N = adv.shape
+    sp = None
+    if stop is not None:
+        stop = np.ascontiguousarray(stop, dtype=np.uint8)
+        sp = stop.ctypes.data
+    counts = np.zeros(3, dtype=np.int64)
+    sumsq = np.zeros(2, dtype=np.float64)
+    _load().sro_batch_stats(adv.ctypes.data, sp, G, N, counts.ctypes.data, sumsq.ctypes.data)
+    return counts, sumsq
+
+
+def savings_fraction(cut: int, n_groups: int, T_max: int, K: int) -> float:
+    return float(_load().sro_savings_fraction(cut, n_groups, T_max, K))
+
+
+def dilution_gain(before: float, after: float) -> float:
+    return float(_load().sro_dilution_gain(before, after))
 
 
 def replay(actions: np.ndarray, upto: int, stride: int = 32):

@@ -155,6 +155,63 @@ void sro_advantage(const float* rewards, const uint8_t* drop_mask, int32_t n_gro
     }
 }
 
+/* Termination fraction tau_K (Appendix B) and the two-clause OR rule (Eq. 3):
+ * Cut = [d_K < d_L] or [tau_K >= tau_H].  A rollout counts as finished by step K when
+ * its `done` flag is set or, without flags, when it has emitted fewer than K actions. */
+void sro_or_rule(const double* mean, const int32_t* lens, const uint8_t* done, int32_t n_groups,
+                 int32_t N, int32_t K, double threshold, double tau_high, double* tau,
+                 uint8_t* stop) {
+    for (int32_t g = 0; g < n_groups; ++g) {
+        int32_t finished = 0;
+        for (int32_t i = 0; i < N; ++i) {
+            const int64_t idx = (int64_t)g * N + i;
+            const int fin = done ? (done[idx] != 0) : (lens[idx] < K);
+            finished += fin ? 1 : 0;
+        }
+        const double t = (double)finished / (double)N;
+        if (tau) tau[g] = t;
+        stop[g] = (mean[g] < threshold || t >= tau_high) ? 1 : 0;
+    }
+}
+
+/* Batch statistics behind the paper's dilution argument (Section 4.5) and its
+ * "gradient signal preserved" figure (Section 3.4): over all trajectories and over the
+ * trajectories of the groups the gate keeps (stop == 0), the number of advantages that
+ * are exactly zero and the sum of squared advantages.
+ * counts: [0] zero advantages, all groups; [1] zero advantages, kept groups;
+ *         [2] kept groups.   sumsq: [0] all groups; [1] kept groups. */
+void sro_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int32_t N,
+                     int64_t* counts, double* sumsq) {
+    counts[0] = counts[1] = counts[2] = 0;
+    sumsq[0] = sumsq[1] = 0.0;
+    for (int32_t g = 0; g < n_groups; ++g) {
+        const int kept = !(stop && stop[g]);
+        counts[2] += kept;
+        for (int32_t i = 0; i < N; ++i) {
+            const double a = (double)adv[(int64_t)g * N + i];
+            const int zero = a == 0.0;
+            counts[0] += zero;
+            sumsq[0] = sumsq[0] + a * a;
+            if (kept) {
+                counts[1] += zero;
+                sumsq[1] = sumsq[1] + a * a;
+            }
+        }
+    }
+}
+
+/* Step-token saving of cutting `cut` of `n_groups` groups at step K of T_max
+ * (caption of Table 1): cut * (T_max - K) / (n_groups * T_max). */
+double sro_savings_fraction(int64_t cut, int64_t n_groups, int32_t T_max, int32_t K) {
+    return (double)(cut * (int64_t)(T_max - K)) / (double)(n_groups * (int64_t)T_max);
+}
+
+/* Predicted gradient-norm gain when the zero-advantage fraction of a batch drops from
+ * `before` to `after` (Section 4.5): (1 - after) / (1 - before). */
+double sro_dilution_gain(double zero_frac_before, double zero_frac_after) {
+    return (1.0 - zero_frac_after) / (1.0 - zero_frac_before);
+}
+
 int32_t sro_max_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();

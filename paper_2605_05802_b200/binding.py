@@ -45,6 +45,10 @@ _SIGNATURES = {
     "sr_incr_init": (ctypes.c_int, [_vp, _sz, _i32, _i32, _i32, _vp]),
     "sr_gate_step_incremental": (ctypes.c_int, [_vp, _sz, _vp, _i32, _i32, _f64, _i32, _vp, _vp, _vp,
                                                 _vp, _vp, _vp]),
+    "sr_gate_or_rule": (ctypes.c_int, [_vp, _vp, _vp, _i32, _i32, _i32, _f64, _f64, _vp, _vp, _vp]),
+    "sr_batch_stats": (ctypes.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp]),
+    "sr_savings_fraction": (ctypes.c_double, [ctypes.c_int64, ctypes.c_int64, _i32, _i32]),
+    "sr_dilution_gain": (ctypes.c_double, [_f64, _f64]),
     "sr_grpo_advantage": (ctypes.c_int, [_vp, _vp, _i32, _i32, _f32, _vp, _vp, _vp]),
     "sr_gate_stages": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
                                       _vp, _vp, _sz, _vp, _vp]),
@@ -199,6 +203,31 @@ def sr_gate_step_incremental(state: torch.Tensor, new_actions: torch.Tensor, thr
         float(threshold), norm_mode, _ptr(pair_dist, torch.int32), _ptr(pair_sum, torch.int32),
         _ptr(mean, torch.float64), _ptr(stop, torch.uint8), _ptr(status, torch.int32),
         _stream(stream)))
+
+
+def sr_gate_or_rule(mean: torch.Tensor, lens: Optional[torch.Tensor], done: Optional[torch.Tensor],
+                    N: int, K: int, threshold: float, tau_high: float, *, tau: Optional[torch.Tensor] = None,
+                    stop: torch.Tensor = None, stream=None) -> None:
+    _check(load().sr_gate_or_rule(_ptr(mean, torch.float64), _ptr(lens, torch.int32),
+                                  _ptr(done, torch.uint8), mean.shape[0], N, K, float(threshold),
+                                  float(tau_high), _ptr(tau, torch.float64), _ptr(stop, torch.uint8),
+                                  _stream(stream)))
+
+
+def sr_batch_stats(adv: torch.Tensor, stop: Optional[torch.Tensor], *, counts: torch.Tensor,
+                   sumsq: torch.Tensor, stream=None) -> None:
+    """counts: int64 [3] device tensor, sumsq: float64 [2] device tensor (see sr_gate.h)."""
+    G, N = adv.shape
+    _check(load().sr_batch_stats(_ptr(adv, torch.float32), _ptr(stop, torch.uint8), G, N,
+                                 _ptr(counts, torch.int64), _ptr(sumsq, torch.float64), _stream(stream)))
+
+
+def sr_savings_fraction(cut: int, n_groups: int, T_max: int, K: int) -> float:
+    return float(load().sr_savings_fraction(cut, n_groups, T_max, K))
+
+
+def sr_dilution_gain(before: float, after: float) -> float:
+    return float(load().sr_dilution_gain(before, after))
 
 
 def sr_grpo_advantage(rewards: torch.Tensor, drop_mask: Optional[torch.Tensor], eps: float, *,

@@ -206,6 +206,33 @@ int sr_gate_step_incremental(void* state, size_t state_bytes, const int32_t* new
                             static_cast<cudaStream_t>(stream));
 }
 
+int sr_gate_or_rule(const double* mean, const int32_t* lens, const uint8_t* done, int32_t n_groups,
+                    int32_t N, int32_t K, double threshold, double tau_high, double* tau,
+                    uint8_t* stop, void* stream) {
+    if (n_groups < 0 || N < 1 || N > SR_MAX_N) return SR_ERR_BAD_N;
+    if (K < 0) return SR_ERR_BAD_K;
+    if (n_groups > 0 && (mean == nullptr || stop == nullptr || (lens == nullptr && done == nullptr)))
+        return SR_ERR_NULL;
+    return launch_or_rule(mean, lens, done, n_groups, N, K, threshold, tau_high, tau, stop,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int sr_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int32_t N,
+                   int64_t* counts, double* sumsq, void* stream) {
+    if (n_groups < 0 || N < 1 || N > SR_MAX_N) return SR_ERR_BAD_N;
+    if (counts == nullptr || sumsq == nullptr || (n_groups > 0 && adv == nullptr)) return SR_ERR_NULL;
+    return launch_batch_stats(adv, stop, n_groups, N, counts, sumsq, static_cast<cudaStream_t>(stream));
+}
+
+double sr_savings_fraction(int64_t cut, int64_t n_groups, int32_t T_max, int32_t K) {
+    if (n_groups <= 0 || T_max <= 0) return 0.0;
+    return (double)(cut * (int64_t)(T_max - K)) / (double)(n_groups * (int64_t)T_max);
+}
+
+double sr_dilution_gain(double zero_frac_before, double zero_frac_after) {
+    return (1.0 - zero_frac_after) / (1.0 - zero_frac_before);
+}
+
 int sr_grpo_advantage(const float* rewards, const uint8_t* drop_mask, int32_t n_groups, int32_t N,
                       float eps, float* adv, uint8_t* zero_var, void* stream) {
     if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;

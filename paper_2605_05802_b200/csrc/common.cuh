@@ -93,4 +93,12 @@ int launch_incr_step(void* state, size_t bytes, const int32_t* new_actions, int3
 int launch_advantage(const float* rewards, const uint8_t* drop_mask, int32_t n_groups, int32_t N,
                      float eps, float* adv, uint8_t* zero_var, cudaStream_t s);
 
+// signals.cu
+int launch_or_rule(const double* mean, const int32_t* lens, const uint8_t* done, int32_t n_groups,
+                   int32_t N, int32_t K, double threshold, double tau_high, double* tau,
+                   uint8_t* stop, cudaStream_t s);
+
+int launch_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int32_t N,
+                       int64_t* counts, double* sumsq, cudaStream_t s);
+
 }  // namespace sr

@@ -94,6 +94,15 @@ def test_incremental_and_advantage_reject_bad_arguments(lib):
     assert step(fake, 1 << 20, None, 4, 8, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_NULL
     assert step(fake, 1 << 20, fake, 4, 8, 0.12, 7, None, None, None, fake, None, None) == binding.SR_ERR_BAD_MODE
     assert step(fake, 16, fake, 4, 8, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_STATE_SIZE
+    orr = lib.sr_gate_or_rule
+    assert orr(None, fake, None, 4, 8, 10, 0.12, 0.9, None, fake, None) == binding.SR_ERR_NULL
+    assert orr(fake, None, None, 4, 8, 10, 0.12, 0.9, None, fake, None) == binding.SR_ERR_NULL
+    assert orr(fake, fake, None, 4, 33, 10, 0.12, 0.9, None, fake, None) == binding.SR_ERR_BAD_N
+    assert orr(None, None, None, 0, 8, 10, 0.12, 0.9, None, None, None) == binding.SR_OK
+    bs = lib.sr_batch_stats
+    assert bs(fake, None, 4, 8, None, fake, None) == binding.SR_ERR_NULL
+    assert bs(None, None, 4, 8, fake, fake, None) == binding.SR_ERR_NULL
+    assert bs(fake, None, 4, 0, fake, fake, None) == binding.SR_ERR_BAD_N
     adv = lib.sr_grpo_advantage
     assert adv(None, None, 4, 8, 1e-6, fake, None, None) == binding.SR_ERR_NULL
     assert adv(fake, None, 4, 1, 1e-6, fake, None, None) == binding.SR_ERR_BAD_N
