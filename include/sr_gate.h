@@ -216,6 +216,30 @@ int sr_grpo_advantage(const float* rewards, const uint8_t* drop_mask, int32_t n_
                       int32_t N, float eps, float* adv, uint8_t* zero_var, void* stream);
 
 /*
+ * sr_group_signals -- the other action-only divergence signals of Appendix B, computed
+ * on the same prefixes as d_K (prefix of rollout i = its first min(len_i, K) actions).
+ * Every output is [n_groups] fp64 and may be NULL.
+ *
+ *   unique_prefix_ratio  distinct prefixes / N (equal = same length, same actions)
+ *   unique_action_ratio  distinct values among the step-K actions a_{i,K}, / N; rollouts
+ *                        that ended before step K share one extra value "no action"
+ *   action_entropy       Shannon entropy of that empirical distribution (natural log)
+ *                        divided by ln N, so that it lies in [0, 1] as Appendix B states
+ *   bigram_jaccard_mean  mean over the pairs (fp64, pair order) of 1 - |A n B| / |A u B|,
+ *                        A, B = the SETS of consecutive action pairs of the two prefixes;
+ *                        a pair of prefixes without any bigram contributes 0
+ *
+ * seqs / lens / stride / K as for sr_gate, with K <= 32 (action-level prefixes).  The
+ * ratios and the Jaccard mean are exact to the last bit of their definition; the entropy
+ * goes through the device logarithm and agrees with a host libm to a few ulp.
+ * (Not computed: obs_unique_ratio, which needs the environment's observations.)
+ */
+int sr_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                     int32_t stride, int32_t K, double* unique_prefix_ratio,
+                     double* unique_action_ratio, double* action_entropy,
+                     double* bigram_jaccard_mean, void* stream);
+
+/*
  * sr_batch_stats -- batch reductions behind two of the paper's figures: the share of
  * zero-advantage trajectories that dilutes the batch-mean loss (Section 4.5: about 40 %
  * without the gate, 28 % with it) and the advantage norm kept after cutting,

@@ -66,6 +66,10 @@ def _load():
         lib.sro_savings_fraction.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32]
         lib.sro_dilution_gain.restype = ctypes.c_double
         lib.sro_dilution_gain.argtypes = [ctypes.c_double, ctypes.c_double]
+        lib.sro_group_signals.restype = None
+        lib.sro_group_signals.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                          ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.c_void_p]
         lib.sro_max_threads.restype = ctypes.c_int32
         _lib = lib
     return _lib
@@ -145,6 +149,20 @@ def or_rule(mean: np.ndarray, lens: Optional[np.ndarray], done: Optional[np.ndar
     _load().sro_or_rule(mean.ctypes.data, lp, dp, G, N, int(K), float(threshold), float(tau_high),
                         tau.ctypes.data, stop.ctypes.data)
     return tau, stop
+
+
+def group_signals(seqs: np.ndarray, lens: Optional[np.ndarray], K: int):
+    """(unique_prefix_ratio, unique_action_ratio, action_entropy, bigram_jaccard_mean),
+    float64 [G] each (Appendix B)."""
+    seqs = np.ascontiguousarray(seqs, dtype=np.int32)
+    G, N, stride = seqs.shape
+    lp = None
+    if lens is not None:
+        lens = np.ascontiguousarray(lens, dtype=np.int32)
+        lp = lens.ctypes.data
+    outs = [np.zeros(G, dtype=np.float64) for _ in range(4)]
+    _load().sro_group_signals(seqs.ctypes.data, lp, G, N, stride, int(K), *[o.ctypes.data for o in outs])
+    return tuple(outs)
 
 
 def batch_stats(adv: np.ndarray, stop: Optional[np.ndarray]):

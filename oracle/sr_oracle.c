@@ -174,6 +174,85 @@ void sro_or_rule(const double* mean, const int32_t* lens, const uint8_t* done, i
     }
 }
 
+/* The other action-only divergence signals of Appendix B, on the same prefixes as d_K
+ * (prefix of rollout i = its first m_i = min(len_i, K) actions).  Each output may be NULL.
+ *   unique_prefix_ratio : distinct prefixes / N (equal = same length and same actions)
+ *   unique_action_ratio : distinct values among the step-K actions a_{i,K} / N; rollouts
+ *                         that ended before step K share one extra value "no action"
+ *   action_entropy      : Shannon entropy of that empirical distribution, natural log,
+ *                         divided by ln N so that it lies in [0, 1]
+ *   bigram_jaccard_mean : mean over pairs of 1 - |A n B| / |A u B|, A and B the SETS of
+ *                         consecutive action pairs of the two prefixes; 0 when both are empty */
+void sro_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                       int32_t stride, int32_t K, double* unique_prefix_ratio,
+                       double* unique_action_ratio, double* action_entropy,
+                       double* bigram_jaccard_mean) {
+    const int64_t P = (int64_t)N * (N - 1) / 2;
+    for (int32_t g = 0; g < n_groups; ++g) {
+        const int32_t* base = seqs + (int64_t)g * N * stride;
+        int distinct_prefix = 0, distinct_action = 0;
+        double entropy = 0.0;
+        for (int32_t i = 0; i < N; ++i) {
+            const int32_t mi = prefix_len(lens, (int64_t)g * N + i, K);
+            const int32_t li = lens ? lens[(int64_t)g * N + i] : K;
+            const int has_i = li >= K && K >= 1;              /* a step-K action exists */
+            int first_prefix = 1, first_action = 1, same_action = 0;
+            for (int32_t j = 0; j < N; ++j) {
+                const int32_t mj = prefix_len(lens, (int64_t)g * N + j, K);
+                const int32_t lj = lens ? lens[(int64_t)g * N + j] : K;
+                const int has_j = lj >= K && K >= 1;
+                int same_p = mi == mj;
+                for (int32_t r = 0; same_p && r < mi; ++r)
+                    if (base[i * stride + r] != base[j * stride + r]) same_p = 0;
+                const int same_a = has_i == has_j &&
+                                   (!has_i || base[i * stride + K - 1] == base[j * stride + K - 1]);
+                if (j < i && same_p) first_prefix = 0;
+                if (j < i && same_a) first_action = 0;
+                same_action += same_a;
+            }
+            distinct_prefix += first_prefix;
+            distinct_action += first_action;
+            if (first_action) {
+                const double pr = (double)same_action / (double)N;
+                entropy = entropy - pr * log(pr);
+            }
+        }
+        if (unique_prefix_ratio) unique_prefix_ratio[g] = (double)distinct_prefix / (double)N;
+        if (unique_action_ratio) unique_action_ratio[g] = (double)distinct_action / (double)N;
+        if (action_entropy) action_entropy[g] = N > 1 ? entropy / log((double)N) : 0.0;
+        if (bigram_jaccard_mean) {
+            double s = 0.0;
+            for (int32_t i = 0; i < N; ++i) {
+                for (int32_t j = i + 1; j < N; ++j) {
+                    const int32_t mi = prefix_len(lens, (int64_t)g * N + i, K);
+                    const int32_t mj = prefix_len(lens, (int64_t)g * N + j, K);
+                    const int32_t* a = base + i * stride;
+                    const int32_t* b = base + j * stride;
+                    int na = 0, nb = 0, both = 0;
+                    for (int32_t t = 0; t + 1 < mi; ++t) {            /* distinct bigrams of a */
+                        int seen = 0;
+                        for (int32_t u = 0; u < t; ++u)
+                            if (a[u] == a[t] && a[u + 1] == a[t + 1]) seen = 1;
+                        if (seen) continue;
+                        ++na;
+                        for (int32_t u = 0; u + 1 < mj; ++u)
+                            if (b[u] == a[t] && b[u + 1] == a[t + 1]) { ++both; break; }
+                    }
+                    for (int32_t t = 0; t + 1 < mj; ++t) {            /* distinct bigrams of b */
+                        int seen = 0;
+                        for (int32_t u = 0; u < t; ++u)
+                            if (b[u] == b[t] && b[u + 1] == b[t + 1]) seen = 1;
+                        nb += !seen;
+                    }
+                    const int uni = na + nb - both;
+                    s = s + (uni > 0 ? 1.0 - (double)both / (double)uni : 0.0);
+                }
+            }
+            bigram_jaccard_mean[g] = s / (double)P;
+        }
+    }
+}
+
 /* Batch statistics behind the paper's dilution argument (Section 4.5) and its
  * "gradient signal preserved" figure (Section 3.4): over all trajectories and over the
  * trajectories of the groups the gate keeps (stop == 0), the number of advantages that

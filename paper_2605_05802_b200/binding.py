@@ -46,6 +46,7 @@ _SIGNATURES = {
     "sr_gate_step_incremental": (ctypes.c_int, [_vp, _sz, _vp, _i32, _i32, _f64, _i32, _vp, _vp, _vp,
                                                 _vp, _vp, _vp]),
     "sr_gate_or_rule": (ctypes.c_int, [_vp, _vp, _vp, _i32, _i32, _i32, _f64, _f64, _vp, _vp, _vp]),
+    "sr_group_signals": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "sr_batch_stats": (ctypes.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp]),
     "sr_savings_fraction": (ctypes.c_double, [ctypes.c_int64, ctypes.c_int64, _i32, _i32]),
     "sr_dilution_gain": (ctypes.c_double, [_f64, _f64]),
@@ -212,6 +213,17 @@ def sr_gate_or_rule(mean: torch.Tensor, lens: Optional[torch.Tensor], done: Opti
                                   _ptr(done, torch.uint8), mean.shape[0], N, K, float(threshold),
                                   float(tau_high), _ptr(tau, torch.float64), _ptr(stop, torch.uint8),
                                   _stream(stream)))
+
+
+def sr_group_signals(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, *,
+                     unique_prefix_ratio=None, unique_action_ratio=None, action_entropy=None,
+                     bigram_jaccard_mean=None, stream=None) -> None:
+    G, N, stride = seqs.shape
+    _check(load().sr_group_signals(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
+                                   _ptr(unique_prefix_ratio, torch.float64),
+                                   _ptr(unique_action_ratio, torch.float64),
+                                   _ptr(action_entropy, torch.float64),
+                                   _ptr(bigram_jaccard_mean, torch.float64), _stream(stream)))
 
 
 def sr_batch_stats(adv: torch.Tensor, stop: Optional[torch.Tensor], *, counts: torch.Tensor,

@@ -217,6 +217,19 @@ int sr_gate_or_rule(const double* mean, const int32_t* lens, const uint8_t* done
                           static_cast<cudaStream_t>(stream));
 }
 
+int sr_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                     int32_t stride, int32_t K, double* unique_prefix_ratio,
+                     double* unique_action_ratio, double* action_entropy,
+                     double* bigram_jaccard_mean, void* stream) {
+    if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;
+    if (stride < 0 || K < 0 || K > stride || K > 32) return SR_ERR_BAD_K;
+    if (n_groups > 0 && seqs == nullptr) return SR_ERR_NULL;
+    if ((stride & 3) != 0 || (reinterpret_cast<uintptr_t>(seqs) & 15) != 0) return SR_ERR_ALIGN;
+    return launch_group_signals(seqs, lens, n_groups, N, stride, K, unique_prefix_ratio,
+                                unique_action_ratio, action_entropy, bigram_jaccard_mean,
+                                static_cast<cudaStream_t>(stream));
+}
+
 int sr_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int32_t N,
                    int64_t* counts, double* sumsq, void* stream) {
     if (n_groups < 0 || N < 1 || N > SR_MAX_N) return SR_ERR_BAD_N;

@@ -98,6 +98,9 @@ int launch_or_rule(const double* mean, const int32_t* lens, const uint8_t* done,
                    int32_t N, int32_t K, double threshold, double tau_high, double* tau,
                    uint8_t* stop, cudaStream_t s);
 
+int launch_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                         int32_t stride, int32_t K, double* upr, double* uar, double* ent,
+                         double* jac, cudaStream_t s);
 int launch_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int32_t N,
                        int64_t* counts, double* sumsq, cudaStream_t s);
 

@@ -153,7 +153,7 @@ __global__ void __launch_bounds__(512, 4)
 incr_step_kernel(IncrArgs a) {
     extern __shared__ __align__(16) unsigned char smem[];
     const int N = a.N, P = pairs_of(N);
-    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int tid = threadIdx.x;
     const int g0 = blockIdx.x * a.gpb;
     const int ng = min(a.gpb, a.n_groups - g0);
     int32_t* s_dist = reinterpret_cast<int32_t*>(smem + a.off_dist);    // [gpb][P]

@@ -99,6 +99,11 @@ def test_incremental_and_advantage_reject_bad_arguments(lib):
     assert orr(fake, None, None, 4, 8, 10, 0.12, 0.9, None, fake, None) == binding.SR_ERR_NULL
     assert orr(fake, fake, None, 4, 33, 10, 0.12, 0.9, None, fake, None) == binding.SR_ERR_BAD_N
     assert orr(None, None, None, 0, 8, 10, 0.12, 0.9, None, None, None) == binding.SR_OK
+    gs = lib.sr_group_signals
+    assert gs(None, None, 4, 8, 32, 10, fake, None, None, None, None) == binding.SR_ERR_NULL
+    assert gs(fake, None, 4, 8, 64, 33, fake, None, None, None, None) == binding.SR_ERR_BAD_K
+    assert gs(fake, None, 4, 1, 32, 10, fake, None, None, None, None) == binding.SR_ERR_BAD_N
+    assert gs(fake + 4, None, 4, 8, 32, 10, fake, None, None, None, None) == binding.SR_ERR_ALIGN
     bs = lib.sr_batch_stats
     assert bs(fake, None, 4, 8, None, fake, None) == binding.SR_ERR_NULL
     assert bs(None, None, 4, 8, fake, fake, None) == binding.SR_ERR_NULL
