@@ -416,6 +416,30 @@ def main():
                                    "hbm_frac": adv_bytes / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         ms = timed(lambda: sr.sr_grpo_advantage(rewards, stop, 1e-6, adv=adv, zero_var=zv), 20)
         extras["advantage_C4"] = {"groups": G, "us_median": statistics.median(ms) * 1e3}
+        # the rows beyond the gate proper: OR rule, Appendix-B signals, batch statistics
+        w3 = W.large_group_gate(n_groups=65536)
+        s3 = torch.from_numpy(w3.seqs).to(dev)
+        outs = [torch.empty(w3.n_groups, dtype=torch.float64, device=dev) for _ in range(4)]
+        ms = timed(lambda: sr.sr_group_signals(s3, None, w3.K, unique_prefix_ratio=outs[0],
+                                               unique_action_ratio=outs[1], action_entropy=outs[2],
+                                               bigram_jaccard_mean=outs[3]), 5)
+        extras["group_signals_C3x16"] = {"groups": w3.n_groups, "N": w3.N, "us_median": statistics.median(ms) * 1e3,
+                                         "groups_per_s": w3.n_groups / (statistics.median(ms) * 1e-3)}
+        l5 = torch.randint(0, 31, (big, 8), dtype=torch.int32, device=dev)
+        m5 = torch.rand(big, dtype=torch.float64, device=dev)
+        t5 = torch.empty(big, dtype=torch.float64, device=dev)
+        ms = timed(lambda: sr.sr_gate_or_rule(m5, l5, None, 8, 15, 0.12, 0.9, tau=t5, stop=z_), 10)
+        med = statistics.median(ms)
+        or_bytes = big * (8 * 4 + 8 + 8 + 1)
+        extras["or_rule_x64"] = {"groups": big, "us_median": med * 1e3, "hbm_gbs": or_bytes / (med * 1e-3) / 1e9,
+                                 "hbm_frac": or_bytes / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        cnt = torch.empty(3, dtype=torch.int64, device=dev)
+        ssq = torch.empty(2, dtype=torch.float64, device=dev)
+        ms = timed(lambda: sr.sr_batch_stats(a_, z_, counts=cnt, sumsq=ssq), 10)
+        med = statistics.median(ms)
+        bs_bytes = big * (8 * 4 + 1)
+        extras["batch_stats_x64"] = {"groups": big, "us_median": med * 1e3, "hbm_gbs": bs_bytes / (med * 1e-3) / 1e9,
+                                     "hbm_frac": bs_bytes / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         line["extras"] = extras
 
         # CPU baseline: the oracle as it stands on this machine's host cores

@@ -126,23 +126,35 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
 // Batch reductions (Section 4.5 dilution, Section 3.4 norm kept): grid-stride over the
 // trajectories, fp64 partial sums per thread, warp shuffles, one atomic per warp.
 __global__ void __launch_bounds__(256)
-batch_stats_kernel(const float* __restrict__ adv, const uint8_t* __restrict__ stop, long long n_traj,
-                   int N, int n_groups, unsigned long long* counts, double* sumsq) {
+batch_stats_kernel(const float* __restrict__ adv, const uint8_t* __restrict__ stop, int N,
+                   int n_groups, bool vec4, unsigned long long* counts, double* sumsq) {
     double ss_all = 0.0, ss_kept = 0.0;
     unsigned z_all = 0, z_kept = 0, kept_groups = 0;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    for (long long t = t0; t < n_traj; t += stride) {
-        const int g = (int)(t / N);
+    const int stride = gridDim.x * blockDim.x;
+    for (int g = blockIdx.x * blockDim.x + threadIdx.x; g < n_groups; g += stride) {   // one group per thread
         const bool kept = !(stop && stop[g]);
-        const double a = (double)__ldg(adv + t);
-        const bool zero = a == 0.0;
-        const double sq = __dmul_rn(a, a);
-        ss_all += sq;
-        z_all += zero;
-        if (kept) { ss_kept += sq; z_kept += zero; }
+        kept_groups += kept;
+        const float* row = adv + (size_t)g * N;
+        double ss = 0.0;
+        unsigned z = 0;
+        if (vec4) {
+            for (int q = 0; q < N / 4; ++q) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(row) + q);
+                const double a0 = v.x, a1 = v.y, a2 = v.z, a3 = v.w;
+                ss += __dmul_rn(a0, a0); ss += __dmul_rn(a1, a1); ss += __dmul_rn(a2, a2); ss += __dmul_rn(a3, a3);
+                z += (a0 == 0.0) + (a1 == 0.0) + (a2 == 0.0) + (a3 == 0.0);
+            }
+        } else {
+            for (int i = 0; i < N; ++i) {
+                const double a = (double)__ldg(row + i);
+                ss += __dmul_rn(a, a);
+                z += a == 0.0;
+            }
+        }
+        ss_all += ss;
+        z_all += z;
+        if (kept) { ss_kept += ss; z_kept += z; }
     }
-    for (long long g = t0; g < n_groups; g += stride) kept_groups += !(stop && stop[g]);
     for (int off = 16; off > 0; off >>= 1) {
         ss_all += __shfl_xor_sync(0xFFFFFFFFu, ss_all, off);
         ss_kept += __shfl_xor_sync(0xFFFFFFFFu, ss_kept, off);
@@ -150,12 +162,27 @@ batch_stats_kernel(const float* __restrict__ adv, const uint8_t* __restrict__ st
         z_kept += __shfl_xor_sync(0xFFFFFFFFu, z_kept, off);
         kept_groups += __shfl_xor_sync(0xFFFFFFFFu, kept_groups, off);
     }
+    // warp results -> shared memory -> one set of atomics per CTA
+    __shared__ double s_ss[2][8];
+    __shared__ unsigned s_cnt[3][8];
+    const int w = threadIdx.x >> 5;
     if ((threadIdx.x & 31) == 0) {
-        atomicAdd(&sumsq[0], ss_all);
-        atomicAdd(&sumsq[1], ss_kept);
-        atomicAdd(&counts[0], (unsigned long long)z_all);
-        atomicAdd(&counts[1], (unsigned long long)z_kept);
-        atomicAdd(&counts[2], (unsigned long long)kept_groups);
+        s_ss[0][w] = ss_all; s_ss[1][w] = ss_kept;
+        s_cnt[0][w] = z_all; s_cnt[1][w] = z_kept; s_cnt[2][w] = kept_groups;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double a = 0.0, k = 0.0;
+        unsigned long long c0 = 0, c1 = 0, c2 = 0;
+        for (int i = 0; i < 8; ++i) {
+            a += s_ss[0][i]; k += s_ss[1][i];
+            c0 += s_cnt[0][i]; c1 += s_cnt[1][i]; c2 += s_cnt[2][i];
+        }
+        atomicAdd(&sumsq[0], a);
+        atomicAdd(&sumsq[1], k);
+        atomicAdd(&counts[0], c0);
+        atomicAdd(&counts[1], c1);
+        atomicAdd(&counts[2], c2);
     }
 }
 
@@ -178,14 +205,14 @@ int launch_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, 
     SR_CUDA_TRY(cudaMemsetAsync(counts, 0, 3 * sizeof(int64_t), s));
     SR_CUDA_TRY(cudaMemsetAsync(sumsq, 0, 2 * sizeof(double), s));
     if (n_groups == 0) return SR_OK;
-    const long long n_traj = (long long)n_groups * N;
     int dev = 0, sms = 0;
     SR_CUDA_TRY(cudaGetDevice(&dev));
     SR_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    long long want = (n_traj + 255) / 256;
-    const long long cap = (long long)sms * 8;
-    const int blocks = (int)(want < cap ? want : cap);
-    batch_stats_kernel<<<blocks, 256, 0, s>>>(adv, stop, n_traj, N, n_groups,
+    const int want = (n_groups + 255) / 256;
+    const int cap = sms * 32;
+    const int blocks = want < cap ? want : cap;
+    const bool vec4 = (N % 4 == 0) && (reinterpret_cast<uintptr_t>(adv) & 15) == 0;
+    batch_stats_kernel<<<blocks, 256, 0, s>>>(adv, stop, N, n_groups, vec4,
                                               reinterpret_cast<unsigned long long*>(counts), sumsq);
     SR_LAUNCH_CHECK("batch_stats_kernel");
     return SR_OK;
