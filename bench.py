@@ -416,6 +416,16 @@ def main():
                                    "hbm_frac": adv_bytes / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         ms = timed(lambda: sr.sr_grpo_advantage(rewards, stop, 1e-6, adv=adv, zero_var=zv), 20)
         extras["advantage_C4"] = {"groups": G, "us_median": statistics.median(ms) * 1e3}
+        # decide mode on the headline workload: same mask, groups dismissed from lower bounds
+        ex = torch.empty(G, dtype=torch.uint8, device=dev)
+        stop_d = torch.empty(G, dtype=torch.uint8, device=dev)
+        ms = timed(lambda: sr.sr_gate_decide(seqs, lens, K, w.threshold, w.norm_mode, pair_sum=ps, mean=mean,
+                                             stop=stop_d, exact=ex, workspace=ws), 20)
+        assert torch.equal(stop_d, stop)
+        extras["decide_C4"] = {"groups": G, "us_median": statistics.median(ms) * 1e3,
+                               "groups_per_s": G / (statistics.median(ms) * 1e-3),
+                               "groups_computed_exactly": int(ex.sum().item()),
+                               "note": "mask-equivalent mode; not the headline (work is skipped by design)"}
         # the rows beyond the gate proper: OR rule, Appendix-B signals, batch statistics
         w3 = W.large_group_gate(n_groups=65536)
         s3 = torch.from_numpy(w3.seqs).to(dev)

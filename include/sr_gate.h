@@ -102,6 +102,31 @@ int sr_gate(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t 
 size_t sr_gate_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
 
 /*
+ * sr_gate_decide -- the same stop mask as sr_gate for less work.  Eq. 2 only consumes the
+ * comparison d_K < d_L, so a group can be dismissed as soon as a LOWER bound of its d_K
+ * reaches the threshold.  For prefixes longer than 32 symbols the match-stream pass
+ * yields such a bound per pair for free: max(|m_i - m_j|, number of symbols of one prefix
+ * that do not occur in the other at all) <= d_ij.  The bounds go through the very same
+ * ordered fp64 sum as the distances (every term is smaller or equal and rounded addition
+ * is monotone), so a group whose bounded d_K is not below the threshold gets stop = 0
+ * without a single column of the recurrence; every other group is computed exactly.
+ *
+ *   stop       identical to sr_gate's, always
+ *   exact      out [n_groups] uint8 or NULL: 1 = pair_dist / pair_sum / mean of the group
+ *              are the exact values (as sr_gate); 0 = they are the lower bounds that
+ *              decided the group (each <= the exact value)
+ *   other arguments and the workspace as for sr_gate (sr_gate_workspace_bytes applies).
+ *
+ * With K <= 32 every group is computed exactly.  The paper has no counterpart; its gate is
+ * evaluated on a handful of groups per iteration and never needed one.
+ */
+int sr_gate_decide(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                   int32_t stride, int32_t K, double threshold, int32_t norm_mode,
+                   int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                   uint8_t* exact, int32_t* status, void* workspace, size_t workspace_bytes,
+                   void* stream);
+
+/*
  * sr_gate_host -- the same computation on HOST buffers: copies seqs/lens to the
  * device, runs sr_gate, and copies the requested outputs back, all enqueued on
  * `stream`; the caller synchronises the stream before reading the outputs.

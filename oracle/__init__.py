@@ -151,6 +151,15 @@ def or_rule(mean: np.ndarray, lens: Optional[np.ndarray], done: Optional[np.ndar
     return tau, stop
 
 
+def absent_lower_bound(a, b) -> int:
+    """max(|len a - len b|, symbols of b that occur nowhere in a): a lower bound of the
+    edit distance (every such symbol must be deleted or substituted)."""
+    a = [int(x) for x in a]
+    b = [int(x) for x in b]
+    present = set(a)
+    return max(abs(len(a) - len(b)), sum(1 for x in b if x not in present))
+
+
 def group_signals(seqs: np.ndarray, lens: Optional[np.ndarray], K: int):
     """(unique_prefix_ratio, unique_action_ratio, action_entropy, bigram_jaccard_mean),
     float64 [G] each (Appendix B)."""

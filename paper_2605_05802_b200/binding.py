@@ -37,6 +37,8 @@ _SIGNATURES = {
     "sr_gate_noalloc": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
                                        _vp, _vp]),
     "sr_gate_noalloc_limit_bytes": (_sz, []),
+    "sr_gate_decide": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp, _vp,
+                                      _vp, _vp, _sz, _vp]),
     "sr_gate_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "sr_gate_host": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
                                     _vp, _vp, _sz, _vp]),
@@ -150,6 +152,20 @@ def sr_gate_noalloc(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, th
                                   _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
                                   _ptr(stop, torch.uint8), _ptr(status, torch.int32),
                                   _stream(stream)))
+
+
+def sr_gate_decide(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, threshold: float,
+                   norm_mode: int = SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None, mean=None,
+                   stop=None, exact=None, status=None, workspace=None, stream=None) -> None:
+    """Same stop mask as sr_gate; groups that a lower bound of d_K already dismisses are
+    not computed (exact[g] = 0 marks them, their other outputs are lower bounds)."""
+    G, N, stride = seqs.shape
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().sr_gate_decide(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
+                                 float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
+                                 _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
+                                 _ptr(stop, torch.uint8), _ptr(exact, torch.uint8),
+                                 _ptr(status, torch.int32), _ptr(workspace), ws_bytes, _stream(stream)))
 
 
 def sr_gate_stages(seqs, lens, K, threshold, norm_mode=SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None,

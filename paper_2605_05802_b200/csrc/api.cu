@@ -97,6 +97,27 @@ int sr_gate(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t 
     return launch_gate_multi(a, workspace, workspace_bytes, s);
 }
 
+int sr_gate_decide(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
+                   int32_t stride, int32_t K, double threshold, int32_t norm_mode,
+                   int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                   uint8_t* exact, int32_t* status, void* workspace, size_t workspace_bytes,
+                   void* stream) {
+    const int rc = check_gate_args(seqs, n_groups, N, stride, K, norm_mode, stop);
+    if (rc != SR_OK) return rc;
+    GateArgs a{seqs, lens, n_groups, N, stride, K, threshold, norm_mode,
+               pair_dist, pair_sum, mean, stop, status};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (K <= 32 || n_groups == 0) {
+        if (exact && n_groups > 0) SR_CUDA_TRY(cudaMemsetAsync(exact, 1, (size_t)n_groups, s));
+        return K <= 32 ? launch_gate_single(a, s) : SR_OK;
+    }
+    const size_t need = gate_multi_workspace_bytes(n_groups, N, stride, K);
+    if (workspace == nullptr || workspace_bytes < need ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255) != 0)
+        return SR_ERR_WORKSPACE;
+    return launch_gate_multi(a, workspace, workspace_bytes, s, nullptr, true, exact);
+}
+
 int sr_gate_stages(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
                    int32_t stride, int32_t K, double threshold, int32_t norm_mode,
                    int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,

@@ -79,8 +79,10 @@ int launch_gate_single(const GateArgs& a, cudaStream_t s);
 size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
 // `ev`: NULL, or 5 events recorded before prep / after prep / after scan+scatter /
 // after dp / after finish.
+// `decide`: finish groups whose lower-bounded d_K already reaches the threshold without
+// running their pairs; `exact` (may be NULL) then receives 1 per group computed exactly.
 int launch_gate_multi(const GateArgs& a, void* ws, size_t ws_bytes, cudaStream_t s,
-                      const cudaEvent_t* ev = nullptr);
+                      const cudaEvent_t* ev = nullptr, bool decide = false, uint8_t* exact = nullptr);
 // incremental.cu
 size_t incr_state_bytes(int32_t n_groups, int32_t N, int32_t max_steps);
 int launch_incr_init(void* state, size_t bytes, int32_t n_groups, int32_t N, int32_t max_steps,

@@ -47,7 +47,7 @@ struct PairDesc {          // 16 bytes
     uint32_t mn;           // m | n << 16
     uint32_t pat_row;      // g * N + pattern rollout
     uint32_t bin;          // bin index; bit 31 = pair needs the dp kernel
-    uint32_t pad;
+    uint32_t lower;        // decide mode: a lower bound of the pair's distance
 };
 
 struct Ctl {               // int32 control block in the workspace
@@ -60,7 +60,7 @@ struct Ctl {               // int32 control block in the workspace
 };
 
 struct MultiWs {
-    size_t off_dist, off_desc, off_loc, off_next, off_order, off_ctl, total;
+    size_t off_dist, off_desc, off_loc, off_next, off_order, off_ctl, off_flag, total;
     int pitch;             // uint16 elements per loc / chain row
 };
 
@@ -70,6 +70,7 @@ MultiWs multi_layout(int32_t n_groups, int32_t N, int32_t K) {
     w.pitch = (K + 7) & ~7;
     size_t off = 0;
     w.off_ctl = off;   off = align_up(off + sizeof(Ctl), 256);
+    w.off_flag = off;  off = align_up(off + (size_t)n_groups, 256);
     w.off_dist = off;  off = align_up(off + (size_t)n_groups * P * 4, 256);
     w.off_desc = off;  off = align_up(off + (size_t)n_groups * P * sizeof(PairDesc), 256);
     w.off_order = off; off = align_up(off + (size_t)n_groups * P * 4, 256);
@@ -142,12 +143,17 @@ __device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, const unsigned l
     return kLocNone;
 }
 
+// kBounds: also count, per text, the columns whose symbol does not occur in the pattern
+// at all.  Each of them costs at least one edit, and so does every unit of length
+// difference: max(|m - n|, absent columns) is a lower bound of the pair's distance that
+// falls out of the look-ups for free.
+template <bool kBounds>
 __global__ void __launch_bounds__(kPrepThreads, 8)
 multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int32_t* dist_out) {
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned long long* s_slot = reinterpret_cast<unsigned long long*>(smem);    // [hslots_max]
     uint32_t* s_next = reinterpret_cast<uint32_t*>(s_slot + hslots_max);         // [pitch]
-    __shared__ int s_txt[SR_MAX_N], s_len[SR_MAX_N], s_qstart[SR_MAX_N + 1], s_ntxt;
+    __shared__ int s_txt[SR_MAX_N], s_len[SR_MAX_N], s_qstart[SR_MAX_N + 1], s_ntxt, s_absent[SR_MAX_N];
 
     const int N = a.N, K = a.K, P = pairs_of(N);
     const int g = blockIdx.x / N, i = blockIdx.x - g * N;
@@ -174,6 +180,7 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
             const int n = clamp_len(a.lens, (size_t)g * N + j, K, neg);
             s_txt[cnt] = j;
             s_len[cnt] = n;
+            s_absent[cnt] = 0;
             s_qstart[cnt] = quads;
             quads += (m > 0) ? (n + 3) >> 2 : 0;
             ++cnt;
@@ -224,21 +231,31 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
         const uint32_t l2 = pattern_lookup(sym.z, s_slot, s_next, hslots, hshift);
         const uint32_t l3 = pattern_lookup(sym.w, s_slot, s_next, hslots, hshift);
         reinterpret_cast<uint2*>(locs + idx * W.pitch)[q] = make_uint2(l0 | (l1 << 16), l2 | (l3 << 16));
+        if (kBounds) {
+            const int left = s_len[t] - 4 * q;           // columns of this quad that exist
+            const int absent = (l0 == kLocNone) + (left > 1 && l1 == kLocNone) +
+                               (left > 2 && l2 == kLocNone) + (left > 3 && l3 == kLocNone);
+            if (absent) atomicAdd(&s_absent[t], absent);
+        }
     }
+    if (kBounds) __syncthreads();
     if (tid < ntxt) {                                 // descriptors, bins, trivial pairs
         const int j = s_txt[tid], n = s_len[tid];
         const int lo = min(i, j), hi = max(i, j);
         const size_t idx = (size_t)g * P + pair_index(lo, hi, N);
         if (m == 0 || n == 0) {
             dist_out[idx] = max(m, n);
-            descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i), 0u, 0u};
+            descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i), 0u,
+                                  (uint32_t)max(m, n)};
         } else {
             int tlog, R;
             team_shape(m, tlog, R);
             const int bin = bin_of(n, tlog, R);
+            const int lower = kBounds ? max(abs(m - n), s_absent[tid]) : 0;
             descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i),
-                                  (uint32_t)bin | 0x80000000u, 0u};
-            atomicAdd(&ctl->hist[bin], 1);
+                                  (uint32_t)bin | 0x80000000u, (uint32_t)lower};
+            if (kBounds) dist_out[idx] = lower;            // the bound kernel bins the pairs it keeps
+            else atomicAdd(&ctl->hist[bin], 1);
         }
     }
     if (neg && tid == 0 && a.status) atomicOr(a.status, SR_STATUS_NEG_LEN);
@@ -456,11 +473,47 @@ multi_dp_kernel(unsigned char* ws, MultiWs W, int32_t* dist_out, uint32_t two) {
     }
 }
 
-// ---------------------------------------------------------------------- finish
+// ----------------------------------------------------------------------- bound
+// Decide mode.  Per group, d_K evaluated on the pairs' lower bounds, in the same order
+// and arithmetic as the real thing: every term is <= the true term and rounded addition
+// is monotone, so the result is <= the true d_K.  If it is already not below the
+// threshold, the gate's answer is "continue" whatever the exact distances are: the
+// group is finished here and its pairs never reach the bit-vector kernel.
 __global__ void __launch_bounds__(128)
-multi_finish_kernel(GateArgs a, const int32_t* dist) {
+multi_bound_kernel(GateArgs a, PairDesc* descs, Ctl* ctl, uint8_t* flag, uint8_t* exact) {
     const int g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= a.n_groups) return;
+    const int N = a.N, P = pairs_of(N);
+    PairDesc* d = descs + (size_t)g * P;
+    double s = 0.0;
+    int isum = 0;
+    for (int p = 0; p < P; ++p) {
+        const int m = (int)(d[p].mn & 0xFFFFu), n = (int)(d[p].mn >> 16);
+        const int lb = (int)d[p].lower;
+        isum += lb;
+        s = __dadd_rn(s, pair_term(lb, m, n, a.norm_mode));      // max(m, n) is symmetric in the roles
+    }
+    const double dk = __ddiv_rn(s, (double)P);
+    const bool open = dk < a.threshold;                  // the bound alone cannot decide
+    flag[g] = open ? 1 : 0;
+    if (exact) exact[g] = open ? 1 : 0;
+    if (open) {
+        for (int p = 0; p < P; ++p)
+            if (d[p].bin & 0x80000000u) atomicAdd(&ctl->hist[d[p].bin & 0x7FFFFFFFu], 1);
+    } else {
+        for (int p = 0; p < P; ++p) d[p].bin &= 0x7FFFFFFFu;
+        if (a.pair_sum) a.pair_sum[g] = isum;
+        if (a.mean) a.mean[g] = dk;
+        a.stop[g] = 0;
+    }
+}
+
+// ---------------------------------------------------------------------- finish
+__global__ void __launch_bounds__(128)
+multi_finish_kernel(GateArgs a, const int32_t* dist, const uint8_t* flag) {
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= a.n_groups) return;
+    if (flag && flag[g] == 0) return;                    // decided from the bounds
     const int N = a.N, P = pairs_of(N);
     bool neg = false;
     double s = 0.0;
@@ -488,7 +541,7 @@ size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, i
 }
 
 int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_t s,
-                      const cudaEvent_t* ev) {
+                      const cudaEvent_t* ev, bool decide, uint8_t* exact) {
     if (a.n_groups == 0) return SR_OK;
     const MultiWs W = multi_layout(a.n_groups, a.N, a.K);
     if (ws_ == nullptr || ws_bytes < W.total || (reinterpret_cast<uintptr_t>(ws_) & 255) != 0)
@@ -507,8 +560,17 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
 
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[0], s));
     SR_CUDA_TRY(cudaMemsetAsync(ctl->hist, 0, sizeof(ctl->hist), s));
-    multi_prep_kernel<<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist);
-    SR_LAUNCH_CHECK("multi_prep_kernel");
+    uint8_t* flag = decide ? ws + W.off_flag : nullptr;
+    if (decide) {
+        multi_prep_kernel<true><<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist);
+        SR_LAUNCH_CHECK("multi_prep_kernel");
+        multi_bound_kernel<<<(a.n_groups + 127) / 128, 128, 0, s>>>(
+            a, reinterpret_cast<PairDesc*>(ws + W.off_desc), ctl, flag, exact);
+        SR_LAUNCH_CHECK("multi_bound_kernel");
+    } else {
+        multi_prep_kernel<false><<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist);
+        SR_LAUNCH_CHECK("multi_prep_kernel");
+    }
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[1], s));
     multi_scan_kernel<<<1, kNumBins, 0, s>>>(ctl);
     SR_LAUNCH_CHECK("multi_scan_kernel");
@@ -531,7 +593,7 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     multi_dp_kernel<<<blocks, kDpWarpsPerCta * 32, 0, s>>>(ws, W, dist, 2u);
     SR_LAUNCH_CHECK("multi_dp_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[3], s));
-    multi_finish_kernel<<<(a.n_groups + 127) / 128, 128, 0, s>>>(a, dist);
+    multi_finish_kernel<<<(a.n_groups + 127) / 128, 128, 0, s>>>(a, dist, flag);
     SR_LAUNCH_CHECK("multi_finish_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[4], s));
     return SR_OK;

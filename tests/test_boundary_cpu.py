@@ -65,6 +65,10 @@ def test_gate_rejects_bad_arguments_before_any_launch(lib):
     assert gate(stride=64, K=64) == binding.SR_ERR_WORKSPACE
     assert gate(stride=64, K=64, ws=fake, wsb=16) == binding.SR_ERR_WORKSPACE
     assert gate(stride=64, K=64, ws=fake + 8, wsb=1 << 30) == binding.SR_ERR_WORKSPACE
+    dec = lib.sr_gate_decide
+    assert dec(fake, None, 4, 8, 64, 64, 0.12, 0, None, None, None, fake, None, None, None, 0, None) == binding.SR_ERR_WORKSPACE
+    assert dec(fake, None, 4, 1, 64, 64, 0.12, 0, None, None, None, fake, None, None, None, 0, None) == binding.SR_ERR_BAD_N
+    assert dec(None, None, 0, 8, 64, 64, 0.12, 0, None, None, None, None, None, None, None, 0, None) == binding.SR_OK
     # an empty batch is a valid no-op on either path
     assert gate(G=0, seqs=None, stop=None) == binding.SR_OK
     assert gate(G=0, seqs=None, stop=None, stride=64, K=64) == binding.SR_OK

@@ -1,0 +1,72 @@
+"""sr_gate_decide: the exact stop mask from lower bounds where they suffice."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2605_05802_b200 import workloads as W
+
+
+def test_absent_symbol_bound_never_exceeds_the_distance():
+    rng = np.random.default_rng(3)
+    for _ in range(400):
+        v = int(rng.integers(2, 12))
+        a = rng.integers(0, v, size=int(rng.integers(0, 40)))
+        b = rng.integers(0, v, size=int(rng.integers(0, 40)))
+        d = oracle.levenshtein(a, b)
+        assert oracle.absent_lower_bound(a, b) <= d
+        assert oracle.absent_lower_bound(b, a) <= d
+    assert oracle.absent_lower_bound([1, 2, 3], [7, 8, 9]) == 3 == oracle.levenshtein([1, 2, 3], [7, 8, 9])
+    assert oracle.absent_lower_bound([1, 2, 3], [3, 2, 1]) == 0
+
+
+def _run_decide(w, thr, norm_mode=0):
+    import torch
+    import paper_2605_05802_b200 as sr
+    dev = torch.device("cuda:0")
+    G, N, stride = w.seqs.shape
+    P = N * (N - 1) // 2
+    seqs = torch.from_numpy(w.seqs).to(dev)
+    lens = torch.from_numpy(w.lens).to(dev)
+    pd = torch.full((G, P), -1, dtype=torch.int32, device=dev)
+    ps = torch.full((G,), -1, dtype=torch.int32, device=dev)
+    mean = torch.full((G,), -1.0, dtype=torch.float64, device=dev)
+    stop = torch.full((G,), 9, dtype=torch.uint8, device=dev)
+    exact = torch.full((G,), 9, dtype=torch.uint8, device=dev)
+    wsb = sr.sr_gate_workspace_bytes(G, N, stride, w.K)
+    ws = torch.empty(max(wsb, 1), dtype=torch.uint8, device=dev) if wsb else None
+    sr.sr_gate_decide(seqs, lens, w.K, thr, norm_mode, pair_dist=pd, pair_sum=ps, mean=mean, stop=stop,
+                      exact=exact, workspace=ws)
+    torch.cuda.synchronize()
+    return [t.cpu().numpy() for t in (pd, ps, mean, stop, exact)]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("thr", [0.05, 0.12, 0.3, 0.6, 0.95])
+def test_decide_mask_is_exact_and_bounds_are_bounds(thr):
+    cases = [W.token_gate(n_groups=48), W.token_gate(seed=8, n_groups=20, min_len=33, max_len=200, N=5),
+             W.agent_gate(K=30)]
+    rng = np.random.default_rng(2)
+    few = W.token_gate(seed=9, n_groups=16, min_len=40, max_len=120, vocab=6)     # heavy repeats
+    cases.append(few)
+    for w in cases:
+        opd, ops, omean, ostop = oracle.gate(w.seqs, w.lens, w.K, thr, w.norm_mode, threads=8)
+        pd, ps, mean, stop, exact = _run_decide(w, thr, w.norm_mode)
+        assert np.array_equal(stop, ostop), w.name                       # the mask, always
+        assert set(np.unique(exact)) <= {0, 1}
+        ex = exact == 1
+        assert np.array_equal(pd[ex], opd[ex]) and np.array_equal(ps[ex], ops[ex])
+        assert np.array_equal(mean[ex].view(np.uint64), omean[ex].view(np.uint64))
+        lo = ~ex                                                          # dismissed from bounds
+        assert (stop[lo] == 0).all()
+        assert (pd[lo] <= opd[lo]).all() and (pd[lo] >= 0).all()
+        assert (ps[lo] == pd[lo].sum(axis=1)).all()
+        assert (mean[lo] <= omean[lo]).all() and (mean[lo] >= thr).all()
+        if w.K <= 32:
+            assert ex.all()
+
+
+@pytest.mark.gpu
+def test_decide_skips_work_on_the_token_workload():
+    w = W.token_gate(n_groups=128)
+    *_, exact = _run_decide(w, 0.12)
+    assert exact.mean() < 0.5          # at the paper's threshold most token-level groups are dismissed early
