@@ -75,6 +75,34 @@ def test_multiword_repeated_symbols_and_ragged_tails():
             assert_gate_matches(got, want, f"multi vocab={vocab} K={K}")
 
 
+def test_multiword_maximum_sizes_and_degenerate_groups():
+    rng = np.random.default_rng(23)
+    # the largest group the ABI accepts at the longest prefix, ragged
+    seqs = rng.integers(0, 50000, size=(2, 32, 1024)).astype(np.int32)
+    seqs[1] = seqs[1, 0]                                   # second group: 32 identical rollouts ...
+    lens = rng.integers(900, 1025, size=(2, 32)).astype(np.int32)
+    lens[1] = 1024                                         # ... of full length: d_K = 0
+    lens[0, 5] = 0
+    lens[0, 6] = 1
+    want = oracle.gate(seqs, lens, 1024, 0.12, threads=8)
+    got = gate_gpu(seqs, lens, 1024, 0.12)
+    assert_gate_matches(got, want, "N=32 K=1024")
+    assert want[2][1] == 0.0 and want[3][1] == 1
+    # K just above the single-word limit, one group, every length 0, one symbol repeated
+    for K, stride in ((33, 36), (64, 64)):
+        seqs = rng.integers(0, 4, size=(1, 4, stride)).astype(np.int32)
+        for lens in (np.zeros((1, 4), dtype=np.int32), np.full((1, 4), K, dtype=np.int32),
+                     np.array([[K, 0, 1, K - 1]], dtype=np.int32)):
+            want = oracle.gate(seqs, lens, K, 0.5)
+            got = gate_gpu(seqs, lens, K, 0.5)
+            assert_gate_matches(got, want, f"K={K} lens={lens.tolist()}")
+    seqs = np.full((3, 3, 256), 7, dtype=np.int32)         # a single symbol: the longest chains
+    lens = np.array([[256, 200, 33], [256, 256, 256], [40, 0, 255]], dtype=np.int32)
+    want = oracle.gate(seqs, lens, 256, 0.3)
+    got = gate_gpu(seqs, lens, 256, 0.3)
+    assert_gate_matches(got, want, "one symbol")
+
+
 @pytest.mark.parametrize("N", [2, 3, 7, 8, 16, 32])
 def test_group_sizes(N):
     rng = np.random.default_rng(N)
