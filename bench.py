@@ -284,9 +284,11 @@ def main():
     d_rew = torch.empty_like(rewards)
     d_stop = torch.empty_like(stop)
 
+    copy_stream = torch.cuda.Stream(device=dev)
+
     def e2e_step():
         sr.sr_gate_host(h_seqs, h_lens, K, w.threshold, w.norm_mode, pair_sum=h_ps, mean=h_mean,
-                        stop=h_stop, arena=arena)
+                        stop=h_stop, arena=arena, copy_stream=copy_stream)
         d_rew.copy_(h_rew, non_blocking=True)
         d_stop.copy_(h_stop, non_blocking=True)      # stream-ordered after the D2H that filled h_stop
         sr.sr_grpo_advantage(d_rew, d_stop, 1e-6, adv=adv, zero_var=zv)

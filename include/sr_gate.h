@@ -134,11 +134,17 @@ int sr_gate_decide(const int32_t* seqs, const int32_t* lens, int32_t n_groups, i
  * asynchronous); outputs that are NULL are not copied.  `arena` is DEVICE scratch
  * of at least sr_gate_host_arena_bytes(...) bytes, 256-byte aligned, used for the
  * staged inputs, outputs and the gate workspace.
+ * `copy_stream` (a second cudaStream_t, or NULL): when given, and different from
+ * `stream`, the inputs are sent in four chunks on it so that the copy of one chunk
+ * overlaps the kernels of the previous one; the outputs still arrive on `stream`, which
+ * is the only stream the caller has to synchronise.  The chunked path creates and
+ * releases a few CUDA events per call (no device memory).
  */
 int sr_gate_host(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
                  int32_t stride, int32_t K, double threshold, int32_t norm_mode,
                  int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
-                 int32_t* status, void* arena, size_t arena_bytes, void* stream);
+                 int32_t* status, void* arena, size_t arena_bytes, void* stream,
+                 void* copy_stream);
 size_t sr_gate_host_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
 
 /*

@@ -41,7 +41,7 @@ _SIGNATURES = {
                                       _vp, _vp, _sz, _vp]),
     "sr_gate_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "sr_gate_host": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
-                                    _vp, _vp, _sz, _vp]),
+                                    _vp, _vp, _sz, _vp, _vp]),
     "sr_gate_host_arena_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "sr_incr_state_bytes": (_sz, [_i32, _i32, _i32]),
     "sr_incr_init": (ctypes.c_int, [_vp, _sz, _i32, _i32, _i32, _vp]),
@@ -188,7 +188,8 @@ def sr_gate_host_arena_bytes(n_groups: int, N: int, stride: int, K: int) -> int:
 
 def sr_gate_host(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, threshold: float,
                  norm_mode: int = SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None, mean=None,
-                 stop=None, status=None, arena: torch.Tensor = None, stream=None) -> None:
+                 stop=None, status=None, arena: torch.Tensor = None, stream=None,
+                 copy_stream: Optional[torch.cuda.Stream] = None) -> None:
     """Same as sr_gate with HOST tensors (ideally pinned) for inputs and outputs and
     a device ``arena``; the caller synchronises the stream before reading outputs."""
     for t in (seqs, lens, pair_dist, pair_sum, mean, stop, status):
@@ -199,7 +200,8 @@ def sr_gate_host(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, thres
                                float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
                                _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
                                _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(arena),
-                               arena.numel() * arena.element_size(), _stream(stream)))
+                               arena.numel() * arena.element_size(), _stream(stream),
+                               None if copy_stream is None else copy_stream.cuda_stream))
 
 
 def sr_incr_state_bytes(n_groups: int, N: int, max_steps: int) -> int:

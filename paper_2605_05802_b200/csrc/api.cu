@@ -156,7 +156,8 @@ size_t sr_gate_host_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int
 int sr_gate_host(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
                  int32_t stride, int32_t K, double threshold, int32_t norm_mode,
                  int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
-                 int32_t* status, void* arena, size_t arena_bytes, void* stream) {
+                 int32_t* status, void* arena, size_t arena_bytes, void* stream,
+                 void* copy_stream) {
     // the alignment rule applies to the device copy, which the arena guarantees
     const int32_t* aligned_stand_in = seqs ? reinterpret_cast<const int32_t*>(uintptr_t(256)) : nullptr;
     int rc = check_gate_args(aligned_stand_in, n_groups, N, stride, K, norm_mode, stop);
@@ -167,23 +168,51 @@ int sr_gate_host(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int
         return SR_ERR_WORKSPACE;
     unsigned char* d = static_cast<unsigned char*>(arena);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
     const size_t P = pairs_of(N);
-    SR_CUDA_TRY(cudaMemcpyAsync(d + h.off_seqs, seqs, (size_t)n_groups * N * stride * 4,
-                                cudaMemcpyHostToDevice, s));
-    if (lens)
-        SR_CUDA_TRY(cudaMemcpyAsync(d + h.off_lens, lens, (size_t)n_groups * N * 4,
-                                    cudaMemcpyHostToDevice, s));
+    // With a copy stream the batch goes over in chunks: the input copy of chunk c+1
+    // overlaps the kernels of chunk c (which run one after the other on `stream` and so
+    // can share the workspace).
+    const bool overlap = cs != nullptr && cs != s && n_groups >= 64;
+    const int chunks = overlap ? 4 : 1;
+    cudaStream_t in_stream = overlap ? cs : s;
     if (status)
         SR_CUDA_TRY(cudaMemcpyAsync(d + h.off_status, status, 4, cudaMemcpyHostToDevice, s));
-    rc = sr_gate(reinterpret_cast<const int32_t*>(d + h.off_seqs),
-                 lens ? reinterpret_cast<const int32_t*>(d + h.off_lens) : nullptr, n_groups, N,
-                 stride, K, threshold, norm_mode,
-                 pair_dist ? reinterpret_cast<int32_t*>(d + h.off_dist) : nullptr,
-                 pair_sum ? reinterpret_cast<int32_t*>(d + h.off_sum) : nullptr,
-                 mean ? reinterpret_cast<double*>(d + h.off_mean) : nullptr, d + h.off_stop,
-                 status ? reinterpret_cast<int32_t*>(d + h.off_status) : nullptr, d + h.off_ws,
-                 h.total - h.off_ws, stream);
-    if (rc != SR_OK) return rc;
+    cudaEvent_t ev = nullptr;
+    if (overlap) {       // the copies must not overtake earlier work on `stream` that uses the arena
+        SR_CUDA_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+        SR_CUDA_TRY(cudaEventRecord(ev, s));
+        SR_CUDA_TRY(cudaStreamWaitEvent(cs, ev, 0));
+        SR_CUDA_TRY(cudaEventDestroy(ev));               // released once it has completed
+    }
+    for (int c = 0; c < chunks; ++c) {
+        const int32_t g0 = (int32_t)((long long)n_groups * c / chunks);
+        const int32_t g1 = (int32_t)((long long)n_groups * (c + 1) / chunks);
+        const int32_t ng = g1 - g0;
+        if (ng == 0) continue;
+        const size_t row0 = (size_t)g0 * N;
+        SR_CUDA_TRY(cudaMemcpyAsync(d + h.off_seqs + row0 * stride * 4, seqs + row0 * stride,
+                                    (size_t)ng * N * stride * 4, cudaMemcpyHostToDevice, in_stream));
+        if (lens)
+            SR_CUDA_TRY(cudaMemcpyAsync(d + h.off_lens + row0 * 4, lens + row0, (size_t)ng * N * 4,
+                                        cudaMemcpyHostToDevice, in_stream));
+        if (overlap) {
+            SR_CUDA_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+            SR_CUDA_TRY(cudaEventRecord(ev, cs));
+            SR_CUDA_TRY(cudaStreamWaitEvent(s, ev, 0));
+            SR_CUDA_TRY(cudaEventDestroy(ev));
+        }
+        rc = sr_gate(reinterpret_cast<const int32_t*>(d + h.off_seqs) + row0 * stride,
+                     lens ? reinterpret_cast<const int32_t*>(d + h.off_lens) + row0 : nullptr, ng, N,
+                     stride, K, threshold, norm_mode,
+                     pair_dist ? reinterpret_cast<int32_t*>(d + h.off_dist) + (size_t)g0 * P : nullptr,
+                     pair_sum ? reinterpret_cast<int32_t*>(d + h.off_sum) + g0 : nullptr,
+                     mean ? reinterpret_cast<double*>(d + h.off_mean) + g0 : nullptr,
+                     d + h.off_stop + g0,
+                     status ? reinterpret_cast<int32_t*>(d + h.off_status) : nullptr, d + h.off_ws,
+                     h.total - h.off_ws, stream);
+        if (rc != SR_OK) return rc;
+    }
     if (pair_dist)
         SR_CUDA_TRY(cudaMemcpyAsync(pair_dist, d + h.off_dist, (size_t)n_groups * P * 4,
                                     cudaMemcpyDeviceToHost, s));

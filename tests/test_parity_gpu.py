@@ -162,7 +162,7 @@ def test_negative_lengths_are_clamped_and_flagged():
 
 def test_host_buffer_entry_point():
     w = W.agent_gate(K=15)
-    for wl in (w, W.token_gate(n_groups=8)):
+    for wl in (w, W.token_gate(n_groups=72)):
         G, N, stride = wl.seqs.shape
         P = N * (N - 1) // 2
         h_seqs = torch.from_numpy(wl.seqs).pin_memory()
@@ -172,10 +172,14 @@ def test_host_buffer_entry_point():
         mean = torch.empty((G,), dtype=torch.float64).pin_memory()
         stop = torch.empty((G,), dtype=torch.uint8).pin_memory()
         arena = torch.empty(sr.sr_gate_host_arena_bytes(G, N, stride, wl.K), dtype=torch.uint8, device="cuda:0")
-        sr.sr_gate_host(h_seqs, h_lens, wl.K, 0.5, pair_dist=pd, pair_sum=ps, mean=mean, stop=stop, arena=arena)
-        torch.cuda.synchronize()
         want = oracle.gate(wl.seqs, wl.lens, wl.K, 0.5, threads=8)
-        assert_gate_matches((pd.numpy(), ps.numpy(), mean.numpy(), stop.numpy()), want, "host " + wl.name)
+        for cs in (None, torch.cuda.Stream()):          # one stream, then copies overlapped in chunks
+            for t in (pd, ps, mean, stop):
+                t.zero_()
+            sr.sr_gate_host(h_seqs, h_lens, wl.K, 0.5, pair_dist=pd, pair_sum=ps, mean=mean, stop=stop,
+                            arena=arena, copy_stream=cs)
+            torch.cuda.synchronize()
+            assert_gate_matches((pd.numpy(), ps.numpy(), mean.numpy(), stop.numpy()), want, "host " + wl.name)
 
 
 # ------------------------------------------------------------------ incremental
