@@ -23,17 +23,26 @@ or_rule_kernel(const double* __restrict__ mean, const int32_t* __restrict__ lens
 }
 
 // The other action-only signals of Appendix B.  One CTA per group: the prefixes are
-// staged once in shared memory (rows of 33 words); one thread per (rollout, position)
-// marks the first occurrence of every bigram of a rollout; one thread per rollout does
-// the prefix / step-K-action comparisons; one thread per pair counts the common bigrams;
-// thread 0 adds everything up in a fixed order.
+// staged once in shared memory (rows of 33 words).  The bigrams of all rollouts are
+// renamed to dense ids through an open-addressing table (as the gate does for symbols),
+// every rollout gets a bit set over those ids, and the Jaccard term of a pair is a few
+// popcounts of AND-ed words instead of K^2 comparisons.  One thread per rollout does
+// the prefix / step-K-action comparisons; thread 0 adds everything up in a fixed order.
+constexpr int kBgSlots = 2048;                  // >= 2 * 32 rollouts * 31 bigrams
+constexpr int kBgWords = 31;                    // 32 * 31 = 992 distinct bigrams at most
+
 __global__ void __launch_bounds__(512)
 group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict__ lens, int N,
-                     int stride, int K, double* upr, double* uar, double* ent, double* jac) {
+                     int stride, int K, int slots, int slot_shift, double* upr, double* uar, double* ent,
+                     double* jac) {
     __shared__ int32_t s_sym[SR_MAX_N * 33];
     __shared__ int32_t s_len[SR_MAX_N], s_raw[SR_MAX_N];
-    __shared__ uint32_t s_first[SR_MAX_N];          // bit t: bigram (t, t+1) is new in its rollout
-    __shared__ int32_t s_fp[SR_MAX_N], s_fa[SR_MAX_N], s_same[SR_MAX_N];
+    __shared__ int32_t s_fp[SR_MAX_N], s_fa[SR_MAX_N], s_same[SR_MAX_N], s_card[SR_MAX_N];
+    __shared__ uint32_t s_owner[kBgSlots];      // element (i * 32 + t) + 1 that claimed the slot
+    __shared__ uint16_t s_bid[kBgSlots];        // dense bigram id of a claimed slot
+    __shared__ uint16_t s_slot[SR_MAX_N * 32];  // slot of every element's bigram
+    __shared__ uint32_t s_bits[SR_MAX_N * kBgWords];
+    __shared__ int s_nbig;
     __shared__ double s_term[SR_MAX_N * (SR_MAX_N - 1) / 2];
     const int g = blockIdx.x, tid = threadIdx.x, nthr = blockDim.x;
     const int P = pairs_of(N);
@@ -41,8 +50,9 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
         const int raw = lens ? lens[(size_t)g * N + i] : K;
         s_raw[i] = raw;
         s_len[i] = min(max(raw, 0), K);
-        s_first[i] = 0u;
+        s_fp[i] = 1; s_fa[i] = 1; s_same[i] = 1;     // every rollout equals itself
     }
+    if (tid == 0) s_nbig = 0;
     const int q4 = (K + 3) >> 2;
     for (int e = tid; e < N * 8; e += nthr) {
         const int i = e >> 3, q = e & 7;
@@ -52,51 +62,65 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
             d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
         }
     }
-    __syncthreads();
-    for (int e = tid; e < N * 32; e += nthr) {
-        const int i = e >> 5, t = e & 31;
-        const int32_t* a = s_sym + i * 33;
-        if (t + 1 < s_len[i]) {
-            bool seen = false;
-            for (int u = 0; u < t; ++u) seen |= (a[u] == a[t]) & (a[u + 1] == a[t + 1]);
-            if (!seen) atomicOr(&s_first[i], 1u << t);
-        }
-    }
-    for (int i = tid; i < N; i += nthr) {
-        const int mi = s_len[i];
-        const bool has_i = s_raw[i] >= K && K >= 1;
-        const int32_t* a = s_sym + i * 33;
-        int first_p = 1, first_a = 1, same_a_cnt = 0;
-        for (int j = 0; j < N; ++j) {
-            const int32_t* b = s_sym + j * 33;
-            bool same_p = mi == s_len[j];
-            for (int r = 0; same_p && r < mi; ++r) same_p = a[r] == b[r];
-            const bool has_j = s_raw[j] >= K && K >= 1;
-            const bool same_a = has_i == has_j && (!has_i || a[K - 1] == b[K - 1]);
-            if (j < i && same_p) first_p = 0;
-            if (j < i && same_a) first_a = 0;
-            same_a_cnt += same_a;
-        }
-        s_fp[i] = first_p; s_fa[i] = first_a; s_same[i] = same_a_cnt;
-    }
-    __syncthreads();
     if (jac) {
+        for (int e = tid; e < slots; e += nthr) s_owner[e] = 0u;
+        for (int e = tid; e < N * kBgWords; e += nthr) s_bits[e] = 0u;
+    }
+    __syncthreads();
+    if (jac) {                                   // bigram (a[t], a[t+1]) of rollout i -> slot
+        for (int e = tid; e < N * 32; e += nthr) {
+            const int i = e >> 5, t = e & 31;
+            if (t + 1 >= s_len[i]) continue;
+            const int32_t x = s_sym[i * 33 + t], y = s_sym[i * 33 + t + 1];
+            uint32_t h = (((uint32_t)x * 0x9E3779B1u) ^ ((uint32_t)y * 0x85EBCA77u)) >> slot_shift;
+            for (int probe = 0; probe < slots; ++probe) {         // at most half of the slots fill up
+                uint32_t o = s_owner[h];
+                if (o == 0u) o = atomicCAS(&s_owner[h], 0u, (uint32_t)e + 1u);
+                if (o == 0u) { s_bid[h] = (uint16_t)atomicAdd(&s_nbig, 1); break; }
+                const int oi = (int)(o - 1u) >> 5, ot = (int)(o - 1u) & 31;
+                if (s_sym[oi * 33 + ot] == x && s_sym[oi * 33 + ot + 1] == y) break;
+                h = (h + 1u) & (uint32_t)(slots - 1);
+            }
+            s_slot[e] = (uint16_t)h;
+        }
+    }
+    // one thread per unordered pair: equal prefixes / equal step-K actions knock out the
+    // later rollout as a "first occurrence" and count towards the action's multiplicity
+    for (int p = tid; p < P; p += nthr) {
+        int i, j;
+        pair_from_index(p, N, i, j);
+        const int32_t* a = s_sym + i * 33;
+        const int32_t* b = s_sym + j * 33;
+        const int mi = s_len[i];
+        bool same_p = mi == s_len[j];
+        for (int r = 0; same_p && r < mi; ++r) same_p = a[r] == b[r];
+        const bool has_i = s_raw[i] >= K && K >= 1, has_j = s_raw[j] >= K && K >= 1;
+        const bool same_a = has_i == has_j && (!has_i || a[K - 1] == b[K - 1]);
+        if (same_p) s_fp[j] = 0;
+        if (same_a) { s_fa[j] = 0; atomicAdd(&s_same[i], 1); atomicAdd(&s_same[j], 1); }
+    }
+    __syncthreads();
+    if (jac) {                                   // bit sets of bigram ids, one per rollout
+        for (int e = tid; e < N * 32; e += nthr) {
+            const int i = e >> 5, t = e & 31;
+            if (t + 1 >= s_len[i]) continue;
+            const uint32_t id = s_bid[s_slot[e]];
+            atomicOr(&s_bits[i * kBgWords + (id >> 5)], 1u << (id & 31));
+        }
+        __syncthreads();
+        const int words = (s_nbig + 31) >> 5;
+        for (int i = tid; i < N; i += nthr) {
+            int c = 0;
+            for (int w = 0; w < words; ++w) c += __popc(s_bits[i * kBgWords + w]);
+            s_card[i] = c;
+        }
+        __syncthreads();
         for (int p = tid; p < P; p += nthr) {
             int i, j;
             pair_from_index(p, N, i, j);
-            const int32_t* a = s_sym + i * 33;
-            const int32_t* b = s_sym + j * 33;
-            const int nbj = s_len[j] - 1;
             int both = 0;
-            uint32_t todo = s_first[i];
-            while (todo) {
-                const int t = __ffs(todo) - 1;
-                todo &= todo - 1;
-                bool hit = false;
-                for (int u = 0; u < nbj; ++u) hit |= (b[u] == a[t]) & (b[u + 1] == a[t + 1]);
-                both += hit;
-            }
-            const int uni = __popc(s_first[i]) + __popc(s_first[j]) - both;
+            for (int w = 0; w < words; ++w) both += __popc(s_bits[i * kBgWords + w] & s_bits[j * kBgWords + w]);
+            const int uni = s_card[i] + s_card[j] - both;
             s_term[p] = uni > 0 ? __dsub_rn(1.0, __ddiv_rn((double)both, (double)uni)) : 0.0;
         }
     }
@@ -195,7 +219,12 @@ int launch_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_gro
     int threads = (max(pairs_of(N), N * 8) + 31) & ~31;
     if (threads < 64) threads = 64;
     if (threads > 512) threads = 512;
-    group_signals_kernel<<<n_groups, threads, 0, s>>>(seqs, lens, N, stride, K, upr, uar, ent, jac);
+    int slots = 64;                                  // >= 2 * N * (K - 1) bigrams, at most kBgSlots
+    while (slots < 2 * N * (K > 1 ? K - 1 : 1)) slots <<= 1;
+    int slot_shift = 32;
+    while ((1 << (32 - slot_shift)) < slots) --slot_shift;
+    group_signals_kernel<<<n_groups, threads, 0, s>>>(seqs, lens, N, stride, K, slots, slot_shift, upr,
+                                                      uar, ent, jac);
     SR_LAUNCH_CHECK("group_signals_kernel");
     return SR_OK;
 }
