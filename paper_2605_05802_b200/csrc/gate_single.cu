@@ -230,10 +230,188 @@ gate_single_kernel(GateArgs a, SingleLayout L) {
     }
 }
 
+// ---------------------------------------------------------------------------------
+// Groups of at most 8 rollouts (28 pairs: the paper's G = 8) fit one warp: lane r owns
+// position r of every prefix during the set-up and pair `lane` during the recurrence,
+// so the whole group is processed with warp-level synchronisation only and the warps
+// of a CTA never wait for one another.  Same steps and tables as the CTA-wide kernel.
+struct WarpLayout {
+    int hslots, hshift, mpitch, kshift;
+    int warp_bytes;                               // shared memory per warp, multiple of 16
+    int sym_off, owner_off, sgid_off;             // build area, phase 1
+    int map_off, peq_off;                         // build area, phase 2 (same bytes)
+    int gid_off, len_off, dist_off, term_off;
+};
+
+constexpr int kWarpsPerCta = 8;
+
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+gate_single_warp_kernel(GateArgs a, WarpLayout L) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int N = a.N, K = a.K, P = pairs_of(N);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = blockIdx.x * kWarpsPerCta + warp;
+    if (g >= a.n_groups) return;                   // whole warps leave; no CTA-wide barrier below
+    unsigned char* base = smem + (size_t)warp * L.warp_bytes;
+    int32_t* s_sym = reinterpret_cast<int32_t*>(base + L.sym_off);        // [N][32]
+    uint32_t* s_owner = reinterpret_cast<uint32_t*>(base + L.owner_off);  // [hslots]
+    uint16_t* s_sgid = reinterpret_cast<uint16_t*>(base + L.sgid_off);    // [hslots]
+    unsigned char* s_map = base + L.map_off;                              // [N][mpitch]
+    uint32_t* s_peq = reinterpret_cast<uint32_t*>(base + L.peq_off);      // [N][33]
+    uint16_t* s_gid = reinterpret_cast<uint16_t*>(base + L.gid_off);      // [N][kGidPitch]
+    int32_t* s_len = reinterpret_cast<int32_t*>(base + L.len_off);        // [8], [8] = id counter
+    int32_t* s_dist = reinterpret_cast<int32_t*>(base + L.dist_off);      // [32]
+    double* s_term = reinterpret_cast<double*>(base + L.term_off);        // [32]
+
+    if (lane < N) {
+        int len = a.lens ? a.lens[(size_t)g * N + lane] : K;
+        if (len < 0) { len = 0; if (a.status) atomicOr(a.status, SR_STATUS_NEG_LEN); }
+        s_len[lane] = min(len, K);
+    }
+    if (lane == 8) s_len[8] = 0;
+    for (int e = lane; e < L.hslots; e += 32) s_owner[e] = 0u;
+    __syncwarp();
+    // Elements (rollout i, position r) are spread over the lanes with r < 2^ks, 2^ks the
+    // power of two >= K: at the paper's K = 10 or 15 a warp covers two rollouts per trip.
+    const int ks = L.kshift, kmask = (1 << ks) - 1, n_elem = N << ks;
+    // ---- symbols (consecutive lanes read consecutive positions of a row)
+    for (int e = lane; e < n_elem; e += 32) {
+        const int i = e >> ks, r = e & kmask;
+        if (r < s_len[i]) s_sym[i * 32 + r] = __ldg(a.seqs + ((size_t)g * N + i) * a.stride + r);
+    }
+    __syncwarp();
+    // ---- dense local ids
+    for (int e = lane; e < n_elem; e += 32) {
+        const int i = e >> ks, r = e & kmask;
+        if (r >= s_len[i]) continue;
+        const int el = i * 32 + r;
+        const int32_t sym = s_sym[el];
+        uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> L.hshift;
+        for (int probe = 0; probe < L.hslots; ++probe) {      // a free or matching slot always exists
+            uint32_t o = s_owner[h];
+            if (o == 0u) o = atomicCAS(&s_owner[h], 0u, (uint32_t)el + 1u);
+            if (o == 0u) { s_sgid[h] = (uint16_t)atomicAdd(&s_len[8], 1); break; }
+            if (s_sym[o - 1u] == sym) break;
+            h = (h + 1u) & (uint32_t)(L.hslots - 1);
+        }
+        s_gid[i * kGidPitch + r] = (uint16_t)h;
+    }
+    __syncwarp();
+    for (int e = lane; e < n_elem; e += 32) {
+        const int i = e >> ks, r = e & kmask;
+        if (r < s_len[i]) s_gid[i * kGidPitch + r] = s_sgid[s_gid[i * kGidPitch + r]];
+    }
+    __syncwarp();
+    // ---- the symbols and the hash table are dead: their bytes become the map and the masks
+    {
+        uint4* init = reinterpret_cast<uint4*>(s_map);
+        const int map_q = L.peq_off >> 4, all_q = (L.peq_off + ((N * kPeqPitch * 4 + 15) & ~15)) >> 4;
+        const uint32_t absent4 = kAbsent * 0x01010101u;
+        for (int e = lane; e < all_q; e += 32)
+            init[e] = e < map_q ? make_uint4(absent4, absent4, absent4, absent4) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncwarp();
+    for (int e = lane; e < n_elem; e += 32) {
+        const int i = e >> ks, r = e & kmask;
+        // several positions with the same symbol store to the same byte; any of them is a
+        // valid representative
+        if (r < s_len[i])
+            reinterpret_cast<volatile unsigned char*>(s_map)[i * L.mpitch + s_gid[i * kGidPitch + r]] = (unsigned char)r;
+    }
+    __syncwarp();
+    for (int e = lane; e < n_elem; e += 32) {
+        const int i = e >> ks, r = e & kmask;
+        if (r < s_len[i]) {
+            const uint32_t rep = s_map[i * L.mpitch + s_gid[i * kGidPitch + r]];
+            atomicOr(&s_peq[i * kPeqPitch + rep], 1u << r);
+        }
+    }
+    __syncwarp();
+    // ---- lane p runs pair p
+    if (lane < P) {
+        int pi, pj;
+        pair_from_index(lane, N, pi, pj);
+        const int mi = s_len[pi], mj = s_len[pj];
+        int mp = mi, mt = mj;
+        if (mj > mi) { const int t = pi; pi = pj; pj = t; mp = mj; mt = mi; }
+        const unsigned char* map = s_map + pi * L.mpitch;
+        const uint32_t* peq = s_peq + pi * kPeqPitch;
+        const uint16_t* txt = s_gid + pj * kGidPitch;
+        uint32_t Pv = 0xFFFFFFFFu, Mv = 0u;
+        for (int c = 0; c < mt; ++c) {
+            const uint32_t Eq = peq[map[txt[c]]];
+            const uint32_t Xv = Eq | Mv;
+            const uint32_t Xh = (((Eq & Pv) + Pv) ^ Pv) | Eq;
+            uint32_t Ph = Mv | ~(Xh | Pv);
+            uint32_t Mh = Pv & Xh;
+            Ph = (Ph << 1) | 1u;
+            Mh = Mh << 1;
+            Pv = Mh | ~(Xv | Ph);
+            Mv = Ph & Xv;
+        }
+        const uint32_t msk = low_mask(mp);
+        const int d = mt + __popc(Pv & msk) - __popc(Mv & msk);
+        s_dist[lane] = d;
+        s_term[lane] = a.norm_mode == SR_NORM_NONE ? (double)d : kQuot.v[d * 33 + mp];
+        if (a.pair_dist) a.pair_dist[(size_t)g * P + lane] = d;
+    }
+    __syncwarp();
+    if (lane == 0) {                              // ordered fp64 sum (Section 3.2), strict gate (Eq. 2)
+        double s = 0.0;
+        int isum = 0, p = 0;
+        for (; p + 4 <= P; p += 4) {
+            const double t0 = s_term[p], t1 = s_term[p + 1], t2 = s_term[p + 2], t3 = s_term[p + 3];
+            isum += s_dist[p] + s_dist[p + 1] + s_dist[p + 2] + s_dist[p + 3];
+            s = __dadd_rn(__dadd_rn(__dadd_rn(__dadd_rn(s, t0), t1), t2), t3);
+        }
+        for (; p < P; ++p) { s = __dadd_rn(s, s_term[p]); isum += s_dist[p]; }
+        const double dk = __ddiv_rn(s, (double)P);
+        if (a.pair_sum) a.pair_sum[g] = isum;
+        if (a.mean) a.mean[g] = dk;
+        a.stop[g] = dk < a.threshold ? 1 : 0;
+    }
+}
+
+int launch_gate_single_warp(const GateArgs& a, cudaStream_t s) {
+    const int N = a.N;
+    WarpLayout L;
+    int h = 32;
+    while (h < 2 * N * a.K) h <<= 1;
+    L.hslots = h;
+    L.hshift = 32;
+    while ((1 << (32 - L.hshift)) < h) --L.hshift;
+    L.kshift = 0;
+    while ((1 << L.kshift) < a.K) ++L.kshift;
+    int mwords = (N * a.K + 3) >> 2;
+    if ((mwords & 1) == 0) ++mwords;
+    L.mpitch = mwords * 4;
+    L.sym_off = 0;
+    L.owner_off = N * 32 * 4;
+    L.sgid_off = L.owner_off + L.hslots * 4;
+    L.map_off = 0;
+    L.peq_off = (N * L.mpitch + 15) & ~15;
+    const int phase1 = L.sgid_off + L.hslots * 2;
+    const int phase2 = L.peq_off + ((N * kPeqPitch * 4 + 15) & ~15);
+    int off = ((phase1 > phase2 ? phase1 : phase2) + 15) & ~15;
+    auto take = [&](int bytes) { int o = off; off = (off + bytes + 15) & ~15; return o; };
+    L.gid_off = take(N * kGidPitch * 2);
+    L.len_off = take(9 * 4);
+    L.dist_off = take(32 * 4);
+    L.term_off = take(32 * 8);
+    L.warp_bytes = off;
+    const int smem = L.warp_bytes * kWarpsPerCta;
+    SR_CUDA_TRY(cudaFuncSetAttribute(gate_single_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int blocks = (a.n_groups + kWarpsPerCta - 1) / kWarpsPerCta;
+    gate_single_warp_kernel<<<blocks, kWarpsPerCta * 32, smem, s>>>(a, L);
+    SR_LAUNCH_CHECK("gate_single_warp_kernel");
+    return SR_OK;
+}
+
 }  // namespace
 
 int launch_gate_single(const GateArgs& a, cudaStream_t s) {
     if (a.n_groups == 0) return SR_OK;
+    if (a.N <= 8) return launch_gate_single_warp(a, s);
     const int N = a.N, P = pairs_of(N);
     SingleLayout L;
     int h = 32;
