@@ -219,7 +219,8 @@ def main():
     G, N, stride, K = w.n_groups, w.N, w.stride, w.K
     P = N * (N - 1) // 2
     cells = W.dp_cells(w.lens, K)
-    wcols = W.word_columns(w.lens, K)
+    wcols_full = W.word_columns(w.lens, K)
+    wcols = W.word_columns(w.lens, K, w.seqs)          # what is left after the pairs' common prefixes
     seqs = torch.from_numpy(w.seqs).to(dev)
     lens = torch.from_numpy(w.lens).to(dev)
     rewards = torch.from_numpy(w.rewards).to(dev)
@@ -323,11 +324,12 @@ def main():
         "clocks": clocks,
         "stage_ms": {"prep": stage_ms[0], "order": stage_ms[1], "dp": stage_ms[2], "finish": stage_ms[3]},
         "roofline": {"kernel": "multi_dp_kernel", "bound": "alu", "achieved": achieved, "peak": alu_peak,
-                     "unit": "Gop/s (int32 lane-ops, 10 per 32-row block per column)",
+                     "unit": "Gop/s (int32 lane-ops, 10 per 32-row block per column, common prefixes of a pair not counted)",
                      "frac": achieved / alu_peak,
                      "peak_basis": f"{sms} SMs x {SM_INT32_LANES} int32 lanes/clk x {peaks['sm_max_mhz']:.0f} MHz (derived)",
                      "traffic": traffic_from_profiles("multi_dp_kernel", os.path.join(ROOT, "paper_2605_05802_b200", "csrc", "gate_multi.cu")),
-                     "word_columns": wcols, "ms_per_launch": dp_ms},
+                     "word_columns": wcols, "word_columns_before_prefix_removal": wcols_full,
+                     "ms_per_launch": dp_ms},
     }
 
     # ------------------------------------------------ side measurements (1 GPU only)
@@ -428,6 +430,30 @@ def main():
                                "groups_per_s": G / (statistics.median(ms) * 1e-3),
                                "groups_computed_exactly": int(ex.sum().item()),
                                "note": "mask-equivalent mode; not the headline (work is skipped by design)"}
+        # the same pipeline on inputs without common prefixes (odd groups diverge from the
+        # first token): nothing is removed, so this line shows the dp kernel on whole matrices
+        w0 = W.token_gate(seed=3, n_groups=args.groups, shared_head=False)
+        s0 = torch.from_numpy(w0.seqs).to(dev)
+        l0 = torch.from_numpy(w0.lens).to(dev)
+        ev0 = []
+        for i in range(20):
+            e5 = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+            for e in e5:
+                e.record()
+            flush_l2(i)
+            sr.sr_gate_stages(s0, l0, K, w0.threshold, w0.norm_mode, pair_sum=ps, mean=mean, stop=stop_d,
+                              workspace=ws, events=e5)
+            ev0.append(e5)
+        torch.cuda.synchronize()
+        dp0 = statistics.median(e5[2].elapsed_time(e5[3]) for e5 in ev0)
+        all0 = statistics.median(e5[0].elapsed_time(e5[4]) for e5 in ev0)
+        wc0 = W.word_columns(w0.lens, K, w0.seqs)
+        extras["C4_no_shared_head"] = {"groups": w0.n_groups, "us_gate": all0 * 1e3, "us_dp": dp0 * 1e3,
+                                       "gcups": W.dp_cells(w0.lens, K) / (all0 * 1e-3) / 1e9,
+                                       "word_columns": wc0, "dp_alu_gops": 10.0 * wc0 / (dp0 * 1e-3) / 1e9,
+                                       "dp_alu_frac": 10.0 * wc0 / (dp0 * 1e-3) / 1e9 / alu_peak}
+        # a large batch of action-level groups at the paper's G = 8, K = 15
+        extras["C2_x128_groups"] = gate_case(W.agent_gate(K=15, n_groups=65536), reps=10)
         # the rows beyond the gate proper: OR rule, Appendix-B signals, batch statistics
         w3 = W.large_group_gate(n_groups=65536)
         s3 = torch.from_numpy(w3.seqs).to(dev)

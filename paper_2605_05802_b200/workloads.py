@@ -183,10 +183,12 @@ def large_group_gate(seed: int = 2, n_groups: int = 4096, threshold: float = 0.1
 
 
 def token_gate(seed: int = 3, n_groups: int = 1024, min_len: int = 256, max_len: int = 1024,
-               N: int = 8, vocab: int = 151936) -> GateWorkload:
+               N: int = 8, vocab: int = 151936, shared_head: bool = True) -> GateWorkload:
     """Token-level prefixes: lengths uniform on min_len..max_len.  Even groups
     are converged (one base, every rollout substitutes an independent random
-    10 % of positions); odd groups share a random-length head then diverge."""
+    10 % of positions); odd groups share a random-length head then diverge
+    (``shared_head=False``: they diverge from the first token, a variant used to
+    time the kernels on inputs without common prefixes)."""
     rng = _rng(seed)
     stride = (max_len + 3) // 4 * 4
     lens = rng.integers(min_len, max_len + 1, size=(n_groups, N)).astype(np.int32)
@@ -195,6 +197,8 @@ def token_gate(seed: int = 3, n_groups: int = 1024, min_len: int = 256, max_len:
     sub = rng.random((n_groups, N, stride)) < 0.10
     conv = np.where(sub, own, base)
     head = (rng.random(n_groups) * (lens.min(axis=1) + 1)).astype(np.int64)
+    if not shared_head:
+        head[:] = 0
     pos = np.arange(stride).reshape(1, 1, stride)
     div = np.where(pos < head.reshape(n_groups, 1, 1), base, own)
     is_conv = (np.arange(n_groups) % 2 == 0).reshape(n_groups, 1, 1)
@@ -264,17 +268,27 @@ def dp_cells(lens: np.ndarray, K: int) -> int:
     return int(((s1 * s1 - s2) // 2).sum())
 
 
-def word_columns(lens: np.ndarray, K: int) -> int:
+def word_columns(lens: np.ndarray, K: int, seqs: np.ndarray = None) -> int:
     """Work units of the bit-vector method: the sum over unordered pairs of
     (text columns) x (32-row blocks of the pattern), taking for every pair the
-    cheaper of the two orientations.  Used only to express roofline fractions."""
+    cheaper of the two orientations.  Used only to express roofline fractions.
+    With ``seqs`` the common prefix of every pair, rounded down to a multiple of
+    four symbols, is left out (nothing at all if one prefix contains the other):
+    the multi-word kernels never run those rows and columns."""
     m = np.minimum(np.maximum(lens.astype(np.int64), 0), K)
-    w = (m + 31) // 32
     total = 0
     N = lens.shape[1]
+    pos = None if seqs is None else np.arange(seqs.shape[2]).reshape(1, -1)
     for i in range(N):
         for j in range(i + 1, N):
-            total += int(np.minimum(m[:, i] * w[:, j], m[:, j] * w[:, i]).sum())
+            a, b = m[:, i], m[:, j]
+            if seqs is not None:
+                lo = np.minimum(a, b)
+                differs = (seqs[:, i, :] != seqs[:, j, :]) | (pos >= lo.reshape(-1, 1))
+                first = np.where(differs.any(axis=1), np.argmax(differs, axis=1), lo)
+                cut = np.where(first >= lo, np.maximum(a, b), first & ~3)
+                a, b = np.maximum(a - cut, 0), np.maximum(b - cut, 0)
+            total += int(np.minimum(a * ((b + 31) // 32), b * ((a + 31) // 32)).sum())
     return total
 
 

@@ -136,3 +136,20 @@ def test_shard_groups_partitions_exactly():
                 assert b == c
             sizes = [b - a for a, b in spans]
             assert max(sizes) - min(sizes) <= 1
+
+
+def test_work_accounting_leaves_out_common_prefixes():
+    """word_columns (the roofline's unit count) with and without the pairs' common prefixes."""
+    import numpy as np
+    from paper_2605_05802_b200 import workloads as W
+    seqs = np.zeros((4, 2, 128), dtype=np.int32)
+    seqs[:, 0, :] = np.arange(128)
+    seqs[:, 1, :] = np.arange(128)
+    seqs[0, 1, 0] = -1            # differ at once: nothing removed
+    seqs[1, 1, 5] = -1            # common prefix 5 -> 4 symbols removed on both sides
+    seqs[2, 1, 100] = -1          # common prefix 100 (a multiple of 4)
+    lens = np.array([[128, 100], [128, 100], [128, 128], [128, 64]], dtype=np.int32)   # last: contained
+    full = [min(100 * 4, 128 * 4), min(100 * 4, 128 * 4), 128 * 4, min(64 * 4, 128 * 2)]
+    assert W.word_columns(lens, 128) == sum(full)
+    cut = [full[0], min(96 * 4, 124 * 3), 28 * 1, 0]
+    assert W.word_columns(lens, 128, seqs) == sum(cut)

@@ -103,6 +103,45 @@ def test_multiword_maximum_sizes_and_degenerate_groups():
     assert_gate_matches(got, want, "one symbol")
 
 
+def test_multiword_shared_prefixes():
+    """Rollouts that agree on their first symbols: the multi-word path leaves the common
+    prefix of a pair out of the recurrence, so every prefix length around its 4-symbol
+    and 128-position steps, whole-prefix containment and repeats on both sides of the
+    cut are compared with the oracle."""
+    rng = np.random.default_rng(31)
+    stride = 512
+    heads = [0, 1, 3, 4, 5, 31, 32, 33, 127, 128, 129, 255, 256, 257, 300, 511]
+    G, N = len(heads), 6
+    for vocab in (5, 300, 100000):                         # small vocabularies: long occurrence chains
+        base = rng.integers(0, vocab, size=(G, 1, stride))
+        own = rng.integers(0, vocab, size=(G, N, stride))
+        pos = np.arange(stride).reshape(1, 1, stride)
+        head = np.array(heads).reshape(G, 1, 1)
+        seqs = np.where(pos < head, base, own).astype(np.int32)
+        # force a mismatch right after the head so that the common prefix is exactly `head`
+        for g, h in enumerate(heads):
+            if h < stride:
+                seqs[g, :, h] = vocab + np.arange(N)
+        lens = rng.integers(40, stride + 1, size=(G, N)).astype(np.int32)
+        lens[:, 0] = stride
+        lens[3, 1] = 2                                     # shorter than the shared head: a pure prefix
+        lens[9, 2] = 128
+        lens[12, 3] = 256
+        lens[15, 4] = 511
+        want = oracle.gate(seqs, lens, stride, 0.5, threads=8)
+        got = gate_gpu(seqs, lens, stride, 0.5)
+        assert_gate_matches(got, want, f"shared heads vocab={vocab}")
+    # identical rollouts of different lengths (every pair: one prefix contains the other),
+    # and rollouts that differ only in their last symbol
+    seqs = np.tile(rng.integers(0, 9, size=(1, 1, 400)), (2, 5, 1)).astype(np.int32)
+    seqs[1, :, 399] = np.arange(5) + 100
+    lens = np.array([[400, 399, 250, 33, 0], [400, 400, 400, 400, 400]], dtype=np.int32)
+    want = oracle.gate(seqs, lens, 400, 0.01)
+    got = gate_gpu(seqs, lens, 400, 0.01)
+    assert_gate_matches(got, want, "contained prefixes")
+    assert want[0][1].max() == 1                           # second group: one substitution per pair
+
+
 @pytest.mark.parametrize("N", [2, 3, 7, 8, 16, 32])
 def test_group_sizes(N):
     rng = np.random.default_rng(N)
