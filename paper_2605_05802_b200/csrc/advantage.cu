@@ -1,8 +1,8 @@
 // Group-relative advantages, Eq. 1 of the paper, with the zero-variance flag of
 // Section 2.1.  One thread per group: the N rewards are read with vector loads,
 // mean and population variance are accumulated in fp64 in index order (explicit
-// round-to-nearest adds and multiplies, no fused multiply-add), and the result is
-// rounded once to fp32.  The kernel moves 8 bytes per rollout plus 1-2 per group and
+// round-to-nearest adds and multiplies, no fused multiply-add), every centred reward is
+// multiplied by the fp64 reciprocal of sigma + eps, and the result is rounded once to fp32.  The kernel moves 8 bytes per rollout plus 1-2 per group and
 // is bound by HBM bandwidth.
 #include "common.cuh"
 
@@ -36,7 +36,7 @@ advantage_kernel(const float* __restrict__ rewards, const uint8_t* __restrict__ 
         if (i < N) equal = equal && (r[i] == r[0]);
     if (zero_var) zero_var[g] = equal ? 1 : 0;
     const bool zero = equal || (drop_mask && drop_mask[g]);
-    double rbar = 0.0, den = 1.0;
+    double rbar = 0.0, inv = 1.0;
     if (!zero) {
         double sum = 0.0;
 #pragma unroll
@@ -50,12 +50,14 @@ advantage_kernel(const float* __restrict__ rewards, const uint8_t* __restrict__ 
                 const double d = __dsub_rn((double)r[i], rbar);
                 ss = __dadd_rn(ss, __dmul_rn(d, d));
             }
-        den = __dadd_rn(__dsqrt_rn(__ddiv_rn(ss, (double)N)), (double)eps);
+        // one reciprocal of sigma + eps, then a multiplication per rollout: the fp64 product is
+        // within one fp64 rounding of the quotient, far inside the fp32 result's own rounding
+        inv = __ddiv_rn(1.0, __dadd_rn(__dsqrt_rn(__ddiv_rn(ss, (double)N)), (double)eps));
     }
     float out[NT > 0 ? NT : SR_MAX_N];
 #pragma unroll
     for (int i = 0; i < (NT > 0 ? NT : SR_MAX_N); ++i)
-        if (i < N) out[i] = zero ? 0.0f : (float)__ddiv_rn(__dsub_rn((double)r[i], rbar), den);
+        if (i < N) out[i] = zero ? 0.0f : (float)__dmul_rn(__dsub_rn((double)r[i], rbar), inv);
     float* dst = adv + (size_t)g * N;
     if (NT > 0 && NT % 4 == 0) {
 #pragma unroll
