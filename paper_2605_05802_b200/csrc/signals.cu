@@ -9,17 +9,26 @@ namespace {
 __global__ void __launch_bounds__(256)
 or_rule_kernel(const double* __restrict__ mean, const int32_t* __restrict__ lens,
                const uint8_t* __restrict__ done, int n_groups, int N, int K, double threshold,
-               double tau_high, double* __restrict__ tau, uint8_t* __restrict__ stop) {
+               double tau_high, bool vec4, double* __restrict__ tau, uint8_t* __restrict__ stop) {
     const int g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= n_groups) return;
+    const double dk = mean[g];
     int finished = 0;
-    for (int i = 0; i < N; ++i) {
-        const size_t idx = (size_t)g * N + i;
-        finished += done ? (done[idx] != 0) : (lens[idx] < K);
+    if (vec4) {                                   // lengths only, rows 16-byte aligned
+        const int4* row = reinterpret_cast<const int4*>(lens + (size_t)g * N);
+        for (int q = 0; q < N / 4; ++q) {
+            const int4 v = __ldg(row + q);
+            finished += (v.x < K) + (v.y < K) + (v.z < K) + (v.w < K);
+        }
+    } else {
+        for (int i = 0; i < N; ++i) {
+            const size_t idx = (size_t)g * N + i;
+            finished += done ? (done[idx] != 0) : (lens[idx] < K);
+        }
     }
     const double t = __ddiv_rn((double)finished, (double)N);
     if (tau) tau[g] = t;
-    stop[g] = (mean[g] < threshold || t >= tau_high) ? 1 : 0;
+    stop[g] = (dk < threshold || t >= tau_high) ? 1 : 0;
 }
 
 // The other action-only signals of Appendix B.  One CTA per group: the prefixes are
@@ -155,7 +164,41 @@ batch_stats_kernel(const float* __restrict__ adv, const uint8_t* __restrict__ st
     double ss_all = 0.0, ss_kept = 0.0;
     unsigned z_all = 0, z_kept = 0, kept_groups = 0;
     const int stride = gridDim.x * blockDim.x;
-    for (int g = blockIdx.x * blockDim.x + threadIdx.x; g < n_groups; g += stride) {   // one group per thread
+    int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (vec4 && N == 8) {
+        // the paper's group size: four groups per trip, their eight 16-byte loads issued
+        // before any arithmetic, zero tests in fp32 (exact), squares in fp64
+        for (; g + 3 * stride < n_groups; g += 4 * stride) {
+            float4 v[4][2];
+            unsigned char st[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float4* row = reinterpret_cast<const float4*>(adv + (size_t)(g + u * stride) * 8);
+                v[u][0] = __ldg(row);
+                v[u][1] = __ldg(row + 1);
+                st[u] = stop ? stop[g + u * stride] : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float f[8] = {v[u][0].x, v[u][0].y, v[u][0].z, v[u][0].w,
+                                    v[u][1].x, v[u][1].y, v[u][1].z, v[u][1].w};
+                double ss = 0.0;
+                unsigned z = 0;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const double a = (double)f[i];
+                    ss += __dmul_rn(a, a);
+                    z += f[i] == 0.0f;
+                }
+                const bool kept = st[u] == 0;
+                kept_groups += kept;
+                ss_all += ss;
+                z_all += z;
+                if (kept) { ss_kept += ss; z_kept += z; }
+            }
+        }
+    }
+    for (; g < n_groups; g += stride) {            // one group per thread and trip
         const bool kept = !(stop && stop[g]);
         kept_groups += kept;
         const float* row = adv + (size_t)g * N;
@@ -238,7 +281,7 @@ int launch_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, 
     SR_CUDA_TRY(cudaGetDevice(&dev));
     SR_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     const int want = (n_groups + 255) / 256;
-    const int cap = sms * 32;
+    const int cap = sms * 16;
     const int blocks = want < cap ? want : cap;
     const bool vec4 = (N % 4 == 0) && (reinterpret_cast<uintptr_t>(adv) & 15) == 0;
     batch_stats_kernel<<<blocks, 256, 0, s>>>(adv, stop, N, n_groups, vec4,
@@ -251,8 +294,9 @@ int launch_or_rule(const double* mean, const int32_t* lens, const uint8_t* done,
                    int32_t N, int32_t K, double threshold, double tau_high, double* tau,
                    uint8_t* stop, cudaStream_t s) {
     if (n_groups == 0) return SR_OK;
+    const bool vec4 = done == nullptr && (N % 4 == 0) && (reinterpret_cast<uintptr_t>(lens) & 15) == 0;
     or_rule_kernel<<<(n_groups + 255) / 256, 256, 0, s>>>(mean, lens, done, n_groups, N, K, threshold,
-                                                          tau_high, tau, stop);
+                                                          tau_high, vec4, tau, stop);
     SR_LAUNCH_CHECK("or_rule_kernel");
     return SR_OK;
 }
