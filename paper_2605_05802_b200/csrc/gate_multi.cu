@@ -558,12 +558,51 @@ multi_bound_kernel(GateArgs a, PairDesc* descs, Ctl* ctl, uint8_t* flag, uint8_t
 }
 
 // ---------------------------------------------------------------------- finish
-__global__ void __launch_bounds__(128)
-multi_finish_kernel(GateArgs a, const int32_t* dist, const uint8_t* flag) {
-    const int g = blockIdx.x * blockDim.x + threadIdx.x;
-    if (g >= a.n_groups) return;
-    if (flag && flag[g] == 0) return;                    // decided from the bounds
+// One thread per pair turns its distance into a term of d_K (the loads and divisions of a
+// group run side by side); one thread per group then adds the terms in pair order.
+constexpr int kFinishThreads = 256;
+
+__global__ void __launch_bounds__(kFinishThreads)
+multi_finish_kernel(GateArgs a, const int32_t* dist, const uint8_t* flag, int gpb) {
+    __shared__ double s_term[kFinishThreads];
+    __shared__ int32_t s_dist[kFinishThreads];
     const int N = a.N, P = pairs_of(N);
+    const int tid = threadIdx.x;
+    const int g0 = blockIdx.x * gpb;
+    const int ng = min(gpb, a.n_groups - g0);
+    if (P <= kFinishThreads) {
+        if (tid < ng * P) {
+            const int g = tid / P, p = tid - g * P;
+            int i, j;
+            pair_from_index(p, N, i, j);
+            bool neg = false;
+            const int mi = clamp_len(a.lens, (size_t)(g0 + g) * N + i, a.K, neg);
+            const int mj = clamp_len(a.lens, (size_t)(g0 + g) * N + j, a.K, neg);
+            const int d = dist[(size_t)g0 * P + tid];
+            s_dist[tid] = d;
+            s_term[tid] = pair_term(d, mi, mj, a.norm_mode);
+        }
+        __syncthreads();
+        if (tid < ng) {
+            const int g = g0 + tid;
+            if (flag && flag[g] == 0) return;                // decided from the bounds
+            double s = 0.0;
+            int isum = 0;
+            for (int p = 0; p < P; ++p) {
+                s = __dadd_rn(s, s_term[tid * P + p]);
+                isum += s_dist[tid * P + p];
+            }
+            const double dk = __ddiv_rn(s, (double)P);
+            if (a.pair_sum) a.pair_sum[g] = isum;
+            if (a.mean) a.mean[g] = dk;
+            a.stop[g] = dk < a.threshold ? 1 : 0;
+        }
+        return;
+    }
+    // groups of more than 23 rollouts (more pairs than threads): one thread per group
+    if (tid != 0) return;
+    const int g = g0;
+    if (flag && flag[g] == 0) return;
     bool neg = false;
     double s = 0.0;
     int isum = 0, p = 0;
@@ -642,7 +681,8 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     multi_dp_kernel<<<blocks, kDpWarpsPerCta * 32, 0, s>>>(ws, W, dist, 2u);
     SR_LAUNCH_CHECK("multi_dp_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[3], s));
-    multi_finish_kernel<<<(a.n_groups + 127) / 128, 128, 0, s>>>(a, dist, flag);
+    const int fin_gpb = P <= kFinishThreads ? kFinishThreads / P : 1;
+    multi_finish_kernel<<<(a.n_groups + fin_gpb - 1) / fin_gpb, kFinishThreads, 0, s>>>(a, dist, flag, fin_gpb);
     SR_LAUNCH_CHECK("multi_finish_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[4], s));
     return SR_OK;
