@@ -90,7 +90,10 @@ const char* sr_last_cuda_error(void);   /* text of the last CUDA failure seen by
  *                  that may overlap on the device need separate workspaces.
  *
  * n_groups == 0 is a valid no-op.  Prefixes of up to 32 symbols use one 32-bit
- * word of bit-parallel state per pair; longer ones use the blocked multi-word path.
+ * word of bit-parallel state per pair; longer ones use the blocked multi-word path,
+ * which leaves the common prefix of a pair out of the computation (the distance of
+ * two sequences equals that of what follows a common prefix), so groups whose
+ * rollouts agree on their first symbols cost less.  Results do not depend on it.
  */
 int sr_gate(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int32_t N,
             int32_t stride, int32_t K, double threshold, int32_t norm_mode,
