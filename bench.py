@@ -273,30 +273,35 @@ def main():
     dp_ms = stage_ms[2]
 
     # ------------------------------------------------------------------ end to end
-    h_seqs = torch.from_numpy(w.seqs).pin_memory()
-    h_lens = torch.from_numpy(w.lens).pin_memory()
+    # host side: the batch as a rollout buffer holds it, prefixes back to back plus row offsets
+    symbols, row_start = W.pack_rows(w.seqs, w.lens)
+    h_sym = torch.from_numpy(symbols).pin_memory()
+    h_rs = torch.from_numpy(row_start).pin_memory()
     h_rew = torch.from_numpy(w.rewards).pin_memory()
     h_ps = torch.empty(G, dtype=torch.int32).pin_memory()
     h_mean = torch.empty(G, dtype=torch.float64).pin_memory()
     h_stop = torch.empty(G, dtype=torch.uint8).pin_memory()
     h_adv = torch.empty((G, N), dtype=torch.float32).pin_memory()
     h_zv = torch.empty(G, dtype=torch.uint8).pin_memory()
-    arena = torch.empty(sr.sr_gate_host_arena_bytes(G, N, stride, K), dtype=torch.uint8, device=dev)
+    arena = torch.empty(sr.sr_gate_host_packed_arena_bytes(G, N, stride, K), dtype=torch.uint8, device=dev)
     d_rew = torch.empty_like(rewards)
     d_stop = torch.empty_like(stop)
 
     copy_stream = torch.cuda.Stream(device=dev)
 
-    def e2e_step():
-        sr.sr_gate_host(h_seqs, h_lens, K, w.threshold, w.norm_mode, pair_sum=h_ps, mean=h_mean,
-                        stop=h_stop, arena=arena, copy_stream=copy_stream)
+    def e2e_tail():
         d_rew.copy_(h_rew, non_blocking=True)
         d_stop.copy_(h_stop, non_blocking=True)      # stream-ordered after the D2H that filled h_stop
         sr.sr_grpo_advantage(d_rew, d_stop, 1e-6, adv=adv, zero_var=zv)
         h_adv.copy_(adv, non_blocking=True)
         h_zv.copy_(zv, non_blocking=True)
 
-    h2d = h_seqs.numel() * 4 + h_lens.numel() * 4 + h_rew.numel() * 4 + h_stop.numel()
+    def e2e_step():
+        sr.sr_gate_host_packed(h_sym, h_rs, N, stride, K, w.threshold, w.norm_mode, pair_sum=h_ps, mean=h_mean,
+                               stop=h_stop, arena=arena)
+        e2e_tail()
+
+    h2d = h_sym.numel() * 4 + h_rs.numel() * 8 + h_rew.numel() * 4 + h_stop.numel()
     d2h = h_ps.numel() * 4 + h_mean.numel() * 8 + h_stop.numel() + h_adv.numel() * 4 + h_zv.numel()
     e2e_ms = sum(timed(e2e_step, args.steps))
     if world > 1:
@@ -319,7 +324,8 @@ def main():
                    "l2": "flushed before every step (256 MiB write + 256 MiB read)", "parallelism": f"groups sharded x{world}, no collective"},
         "groups_per_s": G * world * args.steps / (total_ms * 1e-3),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms / args.steps},
+                "ms_per_step": e2e_ms / args.steps,
+                "input": "packed prefixes + int64 row offsets in pinned host memory (sr_gate_host_packed)"},
         "gpu_launches": 6 * args.steps,
         "clocks": clocks,
         "stage_ms": {"prep": stage_ms[0], "order": stage_ms[1], "dp": stage_ms[2], "finish": stage_ms[3]},
@@ -430,6 +436,19 @@ def main():
                                "groups_per_s": G / (statistics.median(ms) * 1e-3),
                                "groups_computed_exactly": int(ex.sum().item()),
                                "note": "mask-equivalent mode; not the headline (work is skipped by design)"}
+        # end to end with the padded [groups][N][stride] host array instead of packed prefixes
+        h_seqs = torch.from_numpy(w.seqs).pin_memory()
+        h_lens = torch.from_numpy(w.lens).pin_memory()
+
+        def e2e_padded():
+            sr.sr_gate_host(h_seqs, h_lens, K, w.threshold, w.norm_mode, pair_sum=h_ps, mean=h_mean,
+                            stop=h_stop, arena=arena, copy_stream=copy_stream)
+            e2e_tail()
+
+        ms = timed(e2e_padded, 20)
+        extras["e2e_padded_input"] = {"ms_per_step": statistics.median(ms),
+                                      "gcups": cells / (statistics.median(ms) * 1e-3) / 1e9,
+                                      "h2d_bytes_per_step": h_seqs.numel() * 4 + h_lens.numel() * 4 + h_rew.numel() * 4 + h_stop.numel()}
         # the same pipeline on inputs without common prefixes (odd groups diverge from the
         # first token): nothing is removed, so this line shows the dp kernel on whole matrices
         w0 = W.token_gate(seed=3, n_groups=args.groups, shared_head=False)

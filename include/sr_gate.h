@@ -41,6 +41,7 @@ extern "C" {
 #define SR_ERR_CUDA (-7)           /* a CUDA call failed; see sr_last_cuda_error() */
 #define SR_ERR_BAD_MODE (-8)       /* unknown norm_mode */
 #define SR_ERR_SCRATCH_LIMIT (-9)  /* sr_gate_noalloc: problem needs more than the built-in scratch */
+#define SR_ERR_BAD_OFFSETS (-10)   /* sr_gate_host_packed: row_start malformed */
 
 /* limits */
 #define SR_MAX_N 32                /* rollouts per group */
@@ -149,6 +150,37 @@ int sr_gate_host(const int32_t* seqs, const int32_t* lens, int32_t n_groups, int
                  int32_t* status, void* arena, size_t arena_bytes, void* stream,
                  void* copy_stream);
 size_t sr_gate_host_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
+
+/*
+ * sr_gate_host_packed -- sr_gate_host for HOST input in packed (ragged) form: the
+ * prefixes of all rollouts one after the other, without padding.  The operation is the
+ * same d_K / stop mask of Section 3.2 and Eq. 2; only the input layout differs.  Token-
+ * level prefixes of very different lengths fill a padded [rows][stride] array to about
+ * two thirds, and over a host link the copy sets the time of a call, so sending only
+ * the symbols that exist is what shortens it.
+ *
+ *   symbols    in  HOST int32: row r (= g * N + i) owns symbols[row_start[r] .. row_start[r+1])
+ *   row_start  in  HOST int64 [n_groups * N + 1], row_start[0] = 0, non-decreasing; the
+ *                  length of row r is row_start[r+1] - row_start[r] (plays the part of
+ *                  lens; a row may be longer than K, only its first K symbols count).
+ *                  Read on the host during the call, and again by the copy engine: keep
+ *                  both arrays unchanged until the stream has passed the call.
+ *   stride         row pitch of the padded device copy: a multiple of 4, >= K; the sum of
+ *                  all lengths must not exceed n_groups * N * stride
+ *   outputs, status, stream: as for sr_gate_host (HOST pointers)
+ *   arena          DEVICE scratch of sr_gate_host_packed_arena_bytes(...) bytes, 256-byte
+ *                  aligned
+ *
+ * Errors (nothing enqueued): as sr_gate_host, and SR_ERR_BAD_OFFSETS for a malformed
+ * row_start.  The batch is sent in one piece (there is no copy stream: the kernels of a
+ * fraction of a token-level batch take nearly as long as those of the whole batch, so
+ * chunks that overlap copy and kernels lose more than they hide).
+ */
+int sr_gate_host_packed(const int32_t* symbols, const int64_t* row_start, int32_t n_groups,
+                        int32_t N, int32_t stride, int32_t K, double threshold, int32_t norm_mode,
+                        int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
+                        int32_t* status, void* arena, size_t arena_bytes, void* stream);
+size_t sr_gate_host_packed_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
 
 /*
  * sr_gate_noalloc -- sr_gate for callers that cannot allocate device memory.  (The

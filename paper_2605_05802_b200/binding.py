@@ -20,6 +20,7 @@ SR_OK = 0
 SR_ERR_NULL, SR_ERR_BAD_N, SR_ERR_BAD_K, SR_ERR_ALIGN = -1, -2, -3, -4
 SR_ERR_STATE_SIZE, SR_ERR_WORKSPACE, SR_ERR_CUDA, SR_ERR_BAD_MODE = -5, -6, -7, -8
 SR_ERR_SCRATCH_LIMIT = -9
+SR_ERR_BAD_OFFSETS = -10
 SR_NORM_MAXLEN, SR_NORM_NONE = 0, 1
 SR_NO_ACTION = -(2 ** 31)
 SR_STATUS_NEG_LEN, SR_STATUS_STEP_OVERFLOW, SR_STATUS_BAD_STATE = 1, 2, 4
@@ -43,6 +44,9 @@ _SIGNATURES = {
     "sr_gate_host": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
                                     _vp, _vp, _sz, _vp, _vp]),
     "sr_gate_host_arena_bytes": (_sz, [_i32, _i32, _i32, _i32]),
+    "sr_gate_host_packed": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
+                                           _vp, _vp, _sz, _vp]),
+    "sr_gate_host_packed_arena_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "sr_incr_state_bytes": (_sz, [_i32, _i32, _i32]),
     "sr_incr_init": (ctypes.c_int, [_vp, _sz, _i32, _i32, _i32, _vp]),
     "sr_gate_step_incremental": (ctypes.c_int, [_vp, _sz, _vp, _i32, _i32, _f64, _i32, _vp, _vp, _vp,
@@ -202,6 +206,30 @@ def sr_gate_host(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, thres
                                _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(arena),
                                arena.numel() * arena.element_size(), _stream(stream),
                                None if copy_stream is None else copy_stream.cuda_stream))
+
+
+def sr_gate_host_packed_arena_bytes(n_groups: int, N: int, stride: int, K: int) -> int:
+    return int(load().sr_gate_host_packed_arena_bytes(n_groups, N, stride, K))
+
+
+def sr_gate_host_packed(symbols: torch.Tensor, row_start: torch.Tensor, N: int, stride: int, K: int,
+                        threshold: float, norm_mode: int = SR_NORM_MAXLEN, *, pair_dist=None,
+                        pair_sum=None, mean=None, stop=None, status=None, arena: torch.Tensor = None,
+                        stream=None) -> None:
+    """sr_gate_host on packed HOST input: ``symbols`` (int32) holds the prefixes of all rows
+    back to back, ``row_start`` (int64, rows + 1 entries, first 0) where each begins."""
+    for t in (symbols, row_start, pair_dist, pair_sum, mean, stop, status):
+        if t is not None and t.is_cuda:
+            raise ValueError("sr_gate_host_packed takes host tensors")
+    rows = row_start.numel() - 1
+    if rows < 0 or rows % N:
+        raise ValueError("row_start needs n_groups * N + 1 entries")
+    _check(load().sr_gate_host_packed(_ptr(symbols, torch.int32), _ptr(row_start, torch.int64),
+                                      rows // N, N, stride, K, float(threshold), norm_mode,
+                                      _ptr(pair_dist, torch.int32), _ptr(pair_sum, torch.int32),
+                                      _ptr(mean, torch.float64), _ptr(stop, torch.uint8),
+                                      _ptr(status, torch.int32), _ptr(arena),
+                                      arena.numel() * arena.element_size(), _stream(stream)))
 
 
 def sr_incr_state_bytes(n_groups: int, N: int, max_steps: int) -> int:

@@ -26,11 +26,7 @@ static int check_gate_args(const int32_t* seqs, int32_t n_groups, int32_t N, int
     return SR_OK;
 }
 
-struct HostArena {
-    size_t off_seqs, off_lens, off_dist, off_sum, off_mean, off_stop, off_status, off_ws, total;
-};
-
-static HostArena host_arena(int32_t n_groups, int32_t N, int32_t stride, int32_t K) {
+HostArena host_arena(int32_t n_groups, int32_t N, int32_t stride, int32_t K) {
     HostArena h;
     const size_t P = pairs_of(N);
     size_t off = 0;
@@ -66,6 +62,7 @@ const char* sr_strerror(int code) {
         case SR_ERR_CUDA: return "a CUDA call failed (see sr_last_cuda_error)";
         case SR_ERR_BAD_MODE: return "unknown norm_mode";
         case SR_ERR_SCRATCH_LIMIT: return "problem needs more scratch than sr_gate_noalloc's built-in array";
+        case SR_ERR_BAD_OFFSETS: return "row_start does not begin at 0, decreases, or exceeds rows x stride symbols";
         default: return "unknown error code";
     }
 }

@@ -73,6 +73,12 @@ __device__ __forceinline__ double pair_term(int d, int mi, int mj, int norm_mode
 
 size_t align_up(size_t x, size_t a);
 
+// Device arena of the host-buffer entry points (api.cu): staged inputs, outputs, gate workspace.
+struct HostArena {
+    size_t off_seqs, off_lens, off_dist, off_sum, off_mean, off_stop, off_status, off_ws, total;
+};
+HostArena host_arena(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
+
 // gate_single.cu: prefixes of at most 32 symbols, one 32-bit word per pair.
 int launch_gate_single(const GateArgs& a, cudaStream_t s);
 // gate_multi.cu: prefixes of up to SR_MAX_K symbols, blocked multi-word.

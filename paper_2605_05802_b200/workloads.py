@@ -292,6 +292,18 @@ def word_columns(lens: np.ndarray, K: int, seqs: np.ndarray = None) -> int:
     return total
 
 
+def pack_rows(seqs: np.ndarray, lens: np.ndarray):
+    """Packed (ragged) form of a padded batch: the first len symbols of every row back to
+    back, and the int64 offsets at which the rows begin (rows + 1 entries)."""
+    G, N, stride = seqs.shape
+    n = np.clip(lens.reshape(-1).astype(np.int64), 0, stride)
+    row_start = np.zeros(G * N + 1, dtype=np.int64)
+    np.cumsum(n, out=row_start[1:])
+    keep = np.arange(stride).reshape(1, stride) < n.reshape(-1, 1)
+    symbols = np.ascontiguousarray(seqs.reshape(G * N, stride)[keep], dtype=np.int32)
+    return symbols, row_start
+
+
 def all_gate_configs() -> List[GateWorkload]:
     return [tiny_gate(), tiny_gate(raw_threshold=False), agent_gate(K=15), agent_gate(K=30),
             large_group_gate(), token_gate()]

@@ -153,3 +153,24 @@ def test_work_accounting_leaves_out_common_prefixes():
     assert W.word_columns(lens, 128) == sum(full)
     cut = [full[0], min(96 * 4, 124 * 3), 28 * 1, 0]
     assert W.word_columns(lens, 128, seqs) == sum(cut)
+
+
+def test_packed_host_entry_rejects_bad_offsets_before_any_launch(lib):
+    import numpy as np
+    sym = np.zeros(64, dtype=np.int32)
+    stop = np.zeros(1, dtype=np.uint8)
+    fn = lib.sr_gate_host_packed
+
+    def call(row_start, stride=32, K=30, n_groups=1, N=2):
+        rs = np.asarray(row_start, dtype=np.int64)
+        return fn(sym.ctypes.data, rs.ctypes.data, n_groups, N, stride, K, 0.5, 0, None, None, None,
+                  stop.ctypes.data, None, None, 0, None)
+
+    assert call([1, 5, 9]) == binding.SR_ERR_BAD_OFFSETS          # does not begin at 0
+    assert call([0, 9, 5]) == binding.SR_ERR_BAD_OFFSETS          # decreases
+    assert call([0, 40, 65]) == binding.SR_ERR_BAD_OFFSETS        # more symbols than rows x stride
+    assert call([0, 5, 9], stride=30) == binding.SR_ERR_BAD_K     # stride not a multiple of 4
+    assert call([0, 5, 9], K=33) == binding.SR_ERR_BAD_K          # K > stride
+    assert call([0, 5, 9]) == binding.SR_ERR_WORKSPACE            # well-formed, but no arena
+    assert call([0], n_groups=0) == binding.SR_OK
+    assert lib.sr_gate_host_packed_arena_bytes(4, 8, 64, 64) > lib.sr_gate_host_arena_bytes(4, 8, 64, 64)
