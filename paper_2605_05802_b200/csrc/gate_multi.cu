@@ -160,6 +160,10 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
     uint32_t* s_next = reinterpret_cast<uint32_t*>(s_slot + hslots_max);         // [pitch]
     __shared__ int s_txt[SR_MAX_N], s_len[SR_MAX_N], s_qstart[SR_MAX_N + 1], s_absent[SR_MAX_N];
     __shared__ int s_cp[SR_MAX_N];
+    // (At K = 1024 the 36 KB of dynamic plus these 528 bytes of static shared memory sit just
+    // under the size at which six CTAs share an SM: 512 bytes more were measured to cost one
+    // CTA per SM and a fifth of the kernel's speed.  Smaller tables with more CTAs per SM are
+    // slower too: the probe length matters more than the residency.)
 
     const int N = a.N, K = a.K, P = pairs_of(N);
     const int g = blockIdx.x / N, i = blockIdx.x - g * N;
