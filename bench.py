@@ -298,7 +298,7 @@ def main():
 
     def e2e_step():
         sr.sr_gate_host_packed(h_sym, h_rs, N, stride, K, w.threshold, w.norm_mode, pair_sum=h_ps, mean=h_mean,
-                               stop=h_stop, arena=arena)
+                               stop=h_stop, arena=arena, copy_stream=copy_stream)
         e2e_tail()
 
     h2d = h_sym.numel() * 4 + h_rs.numel() * 8 + h_rew.numel() * 4 + h_stop.numel()
@@ -325,7 +325,8 @@ def main():
         "groups_per_s": G * world * args.steps / (total_ms * 1e-3),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / args.steps,
-                "input": "packed prefixes + int64 row offsets in pinned host memory (sr_gate_host_packed)"},
+                "input": "packed prefixes + int64 row offsets in pinned host memory (sr_gate_host_packed), "
+                         "sent in four pieces on a copy stream under the per-group pass; one recurrence launch"},
         "gpu_launches": 6 * args.steps,
         "clocks": clocks,
         "stage_ms": {"prep": stage_ms[0], "order": stage_ms[1], "dp": stage_ms[2], "finish": stage_ms[3]},

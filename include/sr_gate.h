@@ -168,18 +168,23 @@ size_t sr_gate_host_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int
  *   stride         row pitch of the padded device copy: a multiple of 4, >= K; the sum of
  *                  all lengths must not exceed n_groups * N * stride
  *   outputs, status, stream: as for sr_gate_host (HOST pointers)
+ *   copy_stream    a second cudaStream_t, or NULL.  When given (and different from `stream`,
+ *                  K > 32, at least 64 groups) the symbols are sent on it in four pieces of
+ *                  whole groups, and the gate's per-group pass runs on each piece while the
+ *                  next one is still on the link; the recurrence runs once over the whole
+ *                  batch.  Outputs arrive on `stream`, the only stream to synchronise.  This
+ *                  path creates and releases a few CUDA events per call (no device memory).
  *   arena          DEVICE scratch of sr_gate_host_packed_arena_bytes(...) bytes, 256-byte
  *                  aligned
  *
  * Errors (nothing enqueued): as sr_gate_host, and SR_ERR_BAD_OFFSETS for a malformed
- * row_start.  The batch is sent in one piece (there is no copy stream: the kernels of a
- * fraction of a token-level batch take nearly as long as those of the whole batch, so
- * chunks that overlap copy and kernels lose more than they hide).
+ * row_start.
  */
 int sr_gate_host_packed(const int32_t* symbols, const int64_t* row_start, int32_t n_groups,
                         int32_t N, int32_t stride, int32_t K, double threshold, int32_t norm_mode,
                         int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
-                        int32_t* status, void* arena, size_t arena_bytes, void* stream);
+                        int32_t* status, void* arena, size_t arena_bytes, void* stream,
+                        void* copy_stream);
 size_t sr_gate_host_packed_arena_bytes(int32_t n_groups, int32_t N, int32_t stride, int32_t K);
 
 /*

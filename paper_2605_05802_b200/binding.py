@@ -45,7 +45,7 @@ _SIGNATURES = {
                                     _vp, _vp, _sz, _vp, _vp]),
     "sr_gate_host_arena_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "sr_gate_host_packed": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _f64, _i32, _vp, _vp, _vp, _vp,
-                                           _vp, _vp, _sz, _vp]),
+                                           _vp, _vp, _sz, _vp, _vp]),
     "sr_gate_host_packed_arena_bytes": (_sz, [_i32, _i32, _i32, _i32]),
     "sr_incr_state_bytes": (_sz, [_i32, _i32, _i32]),
     "sr_incr_init": (ctypes.c_int, [_vp, _sz, _i32, _i32, _i32, _vp]),
@@ -215,7 +215,7 @@ def sr_gate_host_packed_arena_bytes(n_groups: int, N: int, stride: int, K: int) 
 def sr_gate_host_packed(symbols: torch.Tensor, row_start: torch.Tensor, N: int, stride: int, K: int,
                         threshold: float, norm_mode: int = SR_NORM_MAXLEN, *, pair_dist=None,
                         pair_sum=None, mean=None, stop=None, status=None, arena: torch.Tensor = None,
-                        stream=None) -> None:
+                        stream=None, copy_stream: Optional[torch.cuda.Stream] = None) -> None:
     """sr_gate_host on packed HOST input: ``symbols`` (int32) holds the prefixes of all rows
     back to back, ``row_start`` (int64, rows + 1 entries, first 0) where each begins."""
     for t in (symbols, row_start, pair_dist, pair_sum, mean, stop, status):
@@ -229,7 +229,8 @@ def sr_gate_host_packed(symbols: torch.Tensor, row_start: torch.Tensor, N: int, 
                                       _ptr(pair_dist, torch.int32), _ptr(pair_sum, torch.int32),
                                       _ptr(mean, torch.float64), _ptr(stop, torch.uint8),
                                       _ptr(status, torch.int32), _ptr(arena),
-                                      arena.numel() * arena.element_size(), _stream(stream)))
+                                      arena.numel() * arena.element_size(), _stream(stream),
+                                      None if copy_stream is None else copy_stream.cuda_stream))
 
 
 def sr_incr_state_bytes(n_groups: int, N: int, max_steps: int) -> int:

@@ -87,8 +87,17 @@ size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, i
 // after dp / after finish.
 // `decide`: finish groups whose lower-bounded d_K already reaches the threshold without
 // running their pairs; `exact` (may be NULL) then receives 1 per group computed exactly.
+// `feed`: NULL, or the groups become ready on the stream in `pieces` pieces: before the
+// per-group pass of piece [g0, g1) is enqueued, `before(ctx, g0, g1, s)` is called to
+// enqueue what makes those groups' inputs valid (a wait on a copy, an unpacking kernel).
+struct GroupFeed {
+    int pieces;
+    int (*before)(void* ctx, int g0, int g1, cudaStream_t s);
+    void* ctx;
+};
 int launch_gate_multi(const GateArgs& a, void* ws, size_t ws_bytes, cudaStream_t s,
-                      const cudaEvent_t* ev = nullptr, bool decide = false, uint8_t* exact = nullptr);
+                      const cudaEvent_t* ev = nullptr, bool decide = false, uint8_t* exact = nullptr,
+                      const GroupFeed* feed = nullptr);
 // incremental.cu
 size_t incr_state_bytes(int32_t n_groups, int32_t N, int32_t max_steps);
 int launch_incr_init(void* state, size_t bytes, int32_t n_groups, int32_t N, int32_t max_steps,

@@ -85,15 +85,6 @@ MultiWs multi_layout(int32_t n_groups, int32_t N, int32_t K) {
     return w;
 }
 
-// Pattern side of pair (a, b), a < b: a round-robin tournament in which every vertex
-// of an odd cycle beats the following half; with N even the last rollout is a text
-// for everyone.  Every pattern gets floor(N/2) texts (N even: N/2 for all but the last).
-__host__ __device__ inline bool first_is_pattern(int a, int b, int N) {
-    const int M = (N & 1) ? N : N - 1;
-    if (b >= M) return true;
-    return (b - a) <= (M - 1) / 2;
-}
-
 __host__ __device__ inline void team_shape(int m, int& tlog, int& R) {
     // T lanes x R blocks per lane >= W blocks of the pattern, with little padding and
     // R large enough to amortise the per-column work that does not depend on R
@@ -131,12 +122,13 @@ __device__ __forceinline__ unsigned long long make_slot(int32_t sym, uint32_t po
     return ((unsigned long long)(uint32_t)sym << 32) | pos_plus_1;
 }
 
-// Position (or chain head) of `sym` in the pattern hashed in shared memory.
-__device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, const unsigned long long* s_slot,
-                                                   const uint32_t* s_next, int hslots, int hshift) {
-    uint32_t h = ((uint32_t)sym * 0x9E3779B1u) >> hshift;
+// Position (or chain head) of `sym` in the pattern hashed in shared memory, given the
+// content `v` of its home slot `h` (read by the caller, so that the first probes of the
+// four look-ups of a quad are in flight together).
+__device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, uint32_t h, unsigned long long v,
+                                                   const unsigned long long* s_slot,
+                                                   const uint32_t* s_next, int hslots) {
     for (int probe = 0; probe < hslots; ++probe) {     // an empty slot always exists
-        const unsigned long long v = s_slot[h];
         const uint32_t o = (uint32_t)v;
         if (o == 0u) break;
         if ((int32_t)(v >> 32) == sym) {
@@ -144,6 +136,7 @@ __device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, const unsigned l
             return s_next[first] == kChainEnd ? first : (kLocMulti | first);
         }
         h = (h + 1u) & (uint32_t)(hslots - 1);
+        v = s_slot[h];
     }
     return kLocNone;
 }
@@ -153,8 +146,8 @@ __device__ __forceinline__ uint32_t pattern_lookup(int32_t sym, const unsigned l
 // difference: max(|m - n|, absent columns) is a lower bound of the pair's distance that
 // falls out of the look-ups for free.
 template <bool kBounds>
-__global__ void __launch_bounds__(kPrepThreads, 8)
-multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int32_t* dist_out) {
+__global__ void __launch_bounds__(kPrepThreads, 6)
+multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int32_t* dist_out, int g_base) {
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned long long* s_slot = reinterpret_cast<unsigned long long*>(smem);    // [hslots_max]
     uint32_t* s_next = reinterpret_cast<uint32_t*>(s_slot + hslots_max);         // [pitch]
@@ -163,10 +156,12 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
     // (At K = 1024 the 36 KB of dynamic plus these 528 bytes of static shared memory sit just
     // under the size at which six CTAs share an SM: 512 bytes more were measured to cost one
     // CTA per SM and a fifth of the kernel's speed.  Smaller tables with more CTAs per SM are
-    // slower too: the probe length matters more than the residency.)
+    // slower too: the probe length matters more than the residency.  Six CTAs of 256 threads
+    // leave 40 registers per thread, which the launch bounds grant: capped at 32 the kernel's
+    // time jumped by 10 % on changes as small as one more parameter.)
 
     const int N = a.N, K = a.K, P = pairs_of(N);
-    const int g = blockIdx.x / N, i = blockIdx.x - g * N;
+    const int g = g_base + blockIdx.x / N, i = blockIdx.x % N;
     const int tid = threadIdx.x;
     const int M = (N & 1) ? N : N - 1;
     if (i >= M) return;                               // the last rollout of an even group is never a pattern
@@ -188,15 +183,19 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
     // after a common prefix is removed, so those rows and columns are never looked up nor
     // run through the recurrence.
     const int32_t* pat = a.seqs + ((size_t)g * N + i) * a.stride;
-    // (every warp walks the tournament rule and keeps the texts that fall to it; a closed
-    // form of the list, walked only by the warps that own a text, measured 9 % slower)
-    int ntxt = 0;
+    // Which rollout of a pair is the pattern follows a round-robin tournament: with M = N
+    // for odd N and N - 1 otherwise, rollout i < M is the pattern against the `half` rollouts
+    // after it (cyclically among the first M) and, for even N, against the last rollout,
+    // which is a text for everyone.  Every pattern so serves floor(N / 2) texts.  In
+    // ascending order the texts of pattern i are: the rollouts more than `half` places
+    // before it, the `half` places after it, and the last rollout of an even group.
+    const int half = (M - 1) / 2;
+    const int n_before = max(0, i - half), n_after = min(i + half, M - 1) - i;
+    const int ntxt = n_before + n_after + ((N & 1) ? 0 : 1);
     {
-        const int lane = tid & 31, warp = tid >> 5;
-        for (int j = 0; j < N; ++j) {
-            if (j == i || first_is_pattern(min(i, j), max(i, j), N) != (i < j)) continue;
-            const int t = ntxt++;
-            if ((t & (kPrepThreads / 32 - 1)) != warp) continue;
+        const int lane = tid & 31;
+        for (int t = tid >> 5; t < ntxt; t += kPrepThreads / 32) {
+            const int j = t < n_before ? t : (t < n_before + n_after ? i + 1 + (t - n_before) : N - 1);
             bool neg_t = false;
             const int n = clamp_len(a.lens, (size_t)g * N + j, K, neg_t);
             const int32_t* txt = a.seqs + ((size_t)g * N + j) * a.stride;
@@ -273,10 +272,13 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
         const int lo = min(i, j), hi = max(i, j);
         const size_t idx = (size_t)g * P + pair_index(lo, hi, N);
         const int4 sym = __ldg(reinterpret_cast<const int4*>(a.seqs + ((size_t)g * N + j) * a.stride) + q);
-        const uint32_t l0 = pattern_lookup(sym.x, s_slot, s_next, hslots, hshift);
-        const uint32_t l1 = pattern_lookup(sym.y, s_slot, s_next, hslots, hshift);
-        const uint32_t l2 = pattern_lookup(sym.z, s_slot, s_next, hslots, hshift);
-        const uint32_t l3 = pattern_lookup(sym.w, s_slot, s_next, hslots, hshift);
+        const uint32_t h0 = ((uint32_t)sym.x * 0x9E3779B1u) >> hshift, h1 = ((uint32_t)sym.y * 0x9E3779B1u) >> hshift;
+        const uint32_t h2 = ((uint32_t)sym.z * 0x9E3779B1u) >> hshift, h3 = ((uint32_t)sym.w * 0x9E3779B1u) >> hshift;
+        const unsigned long long v0 = s_slot[h0], v1 = s_slot[h1], v2 = s_slot[h2], v3 = s_slot[h3];
+        const uint32_t l0 = pattern_lookup(sym.x, h0, v0, s_slot, s_next, hslots);
+        const uint32_t l1 = pattern_lookup(sym.y, h1, v1, s_slot, s_next, hslots);
+        const uint32_t l2 = pattern_lookup(sym.z, h2, v2, s_slot, s_next, hslots);
+        const uint32_t l3 = pattern_lookup(sym.w, h3, v3, s_slot, s_next, hslots);
         reinterpret_cast<uint2*>(locs + idx * W.pitch)[q] = make_uint2(l0 | (l1 << 16), l2 | (l3 << 16));
         if (kBounds) {
             const int left = s_len[t] - 4 * q;           // columns of this quad that exist
@@ -633,7 +635,7 @@ size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, i
 }
 
 int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_t s,
-                      const cudaEvent_t* ev, bool decide, uint8_t* exact) {
+                      const cudaEvent_t* ev, bool decide, uint8_t* exact, const GroupFeed* feed) {
     if (a.n_groups == 0) return SR_OK;
     const MultiWs W = multi_layout(a.n_groups, a.N, a.K);
     if (ws_ == nullptr || ws_bytes < W.total || (reinterpret_cast<uintptr_t>(ws_) & 255) != 0)
@@ -653,15 +655,27 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[0], s));
     SR_CUDA_TRY(cudaMemsetAsync(ctl->hist, 0, sizeof(ctl->hist), s));
     uint8_t* flag = decide ? ws + W.off_flag : nullptr;
-    if (decide) {
-        multi_prep_kernel<true><<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist);
+    // The match-stream pass works group by group, so when the groups arrive in pieces it runs
+    // piece by piece: `feed->before` enqueues whatever makes groups [g0, g1) ready on `s`.
+    const int pieces = feed ? feed->pieces : 1;
+    for (int c = 0; c < pieces; ++c) {
+        const int g0 = (int)((long long)a.n_groups * c / pieces);
+        const int g1 = (int)((long long)a.n_groups * (c + 1) / pieces);
+        if (g1 == g0) continue;
+        if (feed) {
+            const int rc = feed->before(feed->ctx, g0, g1, s);
+            if (rc != SR_OK) return rc;
+        }
+        if (decide)
+            multi_prep_kernel<true><<<(g1 - g0) * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist, g0);
+        else
+            multi_prep_kernel<false><<<(g1 - g0) * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist, g0);
         SR_LAUNCH_CHECK("multi_prep_kernel");
+    }
+    if (decide) {
         multi_bound_kernel<<<(a.n_groups + 127) / 128, 128, 0, s>>>(
             a, reinterpret_cast<PairDesc*>(ws + W.off_desc), ctl, flag, exact);
         SR_LAUNCH_CHECK("multi_bound_kernel");
-    } else {
-        multi_prep_kernel<false><<<a.n_groups * a.N, kPrepThreads, prep_smem, s>>>(a, ws, W, hslots, dist);
-        SR_LAUNCH_CHECK("multi_prep_kernel");
     }
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[1], s));
     multi_scan_kernel<<<1, kNumBins, 0, s>>>(ctl);

@@ -28,6 +28,36 @@ unpack_rows_kernel(const int32_t* __restrict__ packed, const long long* __restri
     if (lane == 0) lens[row] = (int)(len < 0x7FFFFFFFLL ? len : 0x7FFFFFFFLL);
 }
 
+// What the pieces of a chunked transfer need on the kernels' stream: wait for the piece's
+// copy, then spread its rows.
+struct FeedCtx {
+    const int32_t* d_packed;
+    const long long* d_start;
+    int32_t* d_seqs;
+    int32_t* d_lens;
+    int N, stride;
+    cudaEvent_t* copied;      // one event per piece, recorded on the copy stream
+    int pieces, n_groups;
+};
+
+int unpack_rows(const FeedCtx& f, int g0, int g1, cudaStream_t s) {
+    const size_t row0 = (size_t)g0 * f.N;
+    const int rows = (g1 - g0) * f.N;
+    unpack_rows_kernel<<<(rows + kUnpackThreads / 32 - 1) / (kUnpackThreads / 32), kUnpackThreads, 0, s>>>(
+        f.d_packed, f.d_start + row0, rows, f.stride, f.d_seqs + row0 * f.stride, f.d_lens + row0);
+    SR_LAUNCH_CHECK("unpack_rows_kernel");
+    return SR_OK;
+}
+
+int feed_piece(void* ctx, int g0, int g1, cudaStream_t s) {
+    const FeedCtx& f = *static_cast<const FeedCtx*>(ctx);
+    // the piece index follows from g0 the same way the pipeline cut the groups
+    int c = 0;
+    while (c + 1 < f.pieces && (int)((long long)f.n_groups * (c + 1) / f.pieces) <= g0) ++c;
+    SR_CUDA_TRY(cudaStreamWaitEvent(s, f.copied[c], 0));
+    return unpack_rows(f, g0, g1, s);
+}
+
 struct PackedArena {
     size_t off_packed, off_start, inner, total;     // `inner`: where the padded-input arena begins
 };
@@ -59,7 +89,8 @@ size_t sr_gate_host_packed_arena_bytes(int32_t n_groups, int32_t N, int32_t stri
 int sr_gate_host_packed(const int32_t* symbols, const int64_t* row_start, int32_t n_groups, int32_t N,
                         int32_t stride, int32_t K, double threshold, int32_t norm_mode,
                         int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
-                        int32_t* status, void* arena, size_t arena_bytes, void* stream) {
+                        int32_t* status, void* arena, size_t arena_bytes, void* stream,
+                        void* copy_stream) {
     if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;
     if (stride < 0 || (stride & 3) || K < 0 || K > stride || K > SR_MAX_K) return SR_ERR_BAD_K;
     if (norm_mode != SR_NORM_MAXLEN && norm_mode != SR_NORM_NONE) return SR_ERR_BAD_MODE;
@@ -88,24 +119,56 @@ int sr_gate_host_packed(const int32_t* symbols, const int64_t* row_start, int32_
     long long* d_start = reinterpret_cast<long long*>(d + pa.off_start);
     int32_t* d_seqs = reinterpret_cast<int32_t*>(di + h.off_seqs);
     int32_t* d_lens = reinterpret_cast<int32_t*>(di + h.off_lens);
-    // The batch goes over in one piece.  Sending it in chunks whose kernels overlap the next
-    // chunk's copy was measured and lost: the kernels of a quarter of a token-level batch take
-    // almost as long as those of the whole batch (a few long pairs set the time of the
-    // recurrence launch), far longer than the quarter's copy.
+    GateArgs ga{d_seqs, d_lens, n_groups, N, stride, K, threshold, norm_mode,
+                pair_dist ? reinterpret_cast<int32_t*>(di + h.off_dist) : nullptr,
+                pair_sum ? reinterpret_cast<int32_t*>(di + h.off_sum) : nullptr,
+                mean ? reinterpret_cast<double*>(di + h.off_mean) : nullptr,
+                di + h.off_stop, status ? reinterpret_cast<int32_t*>(di + h.off_status) : nullptr};
+    FeedCtx f{d_packed, d_start, d_seqs, d_lens, N, stride, nullptr, 1, n_groups};
     if (status) SR_CUDA_TRY(cudaMemcpyAsync(di + h.off_status, status, 4, cudaMemcpyHostToDevice, s));
-    SR_CUDA_TRY(cudaMemcpyAsync(d_start, row_start, (rows + 1) * 8, cudaMemcpyHostToDevice, s));
-    if (total > 0)
-        SR_CUDA_TRY(cudaMemcpyAsync(d_packed, symbols, (size_t)total * 4, cudaMemcpyHostToDevice, s));
-    unpack_rows_kernel<<<(int)((rows + kUnpackThreads / 32 - 1) / (kUnpackThreads / 32)), kUnpackThreads, 0, s>>>(
-        d_packed, d_start, (int)rows, stride, d_seqs, d_lens);
-    SR_LAUNCH_CHECK("unpack_rows_kernel");
-    const int rc = sr_gate(d_seqs, d_lens, n_groups, N, stride, K, threshold, norm_mode,
-                           pair_dist ? reinterpret_cast<int32_t*>(di + h.off_dist) : nullptr,
-                           pair_sum ? reinterpret_cast<int32_t*>(di + h.off_sum) : nullptr,
-                           mean ? reinterpret_cast<double*>(di + h.off_mean) : nullptr,
-                           di + h.off_stop, status ? reinterpret_cast<int32_t*>(di + h.off_status) : nullptr,
-                           di + h.off_ws, h.total - h.off_ws, stream);
-    if (rc != SR_OK) return rc;
+    cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
+    // With a copy stream and long prefixes the symbols go over in four pieces of whole groups
+    // and the per-group pass of the gate (match streams) runs on each piece while the next one
+    // is still on the link; the recurrence then runs ONCE over the whole batch.  Cutting the
+    // whole gate into pieces was measured and lost: the kernels of a quarter of a token-level
+    // batch take almost as long as those of the whole batch, because a few long pairs set the
+    // time of the recurrence launch.
+    if (cs != nullptr && cs != s && K > 32 && n_groups >= 64) {
+        constexpr int kPieces = 4;
+        cudaEvent_t copied[kPieces];
+        cudaEvent_t ev = nullptr;
+        // the copies must not overtake earlier work on `stream` that uses the arena
+        SR_CUDA_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+        SR_CUDA_TRY(cudaEventRecord(ev, s));
+        SR_CUDA_TRY(cudaStreamWaitEvent(cs, ev, 0));
+        SR_CUDA_TRY(cudaEventDestroy(ev));               // released once it has completed
+        SR_CUDA_TRY(cudaMemcpyAsync(d_start, row_start, (rows + 1) * 8, cudaMemcpyHostToDevice, cs));
+        for (int c = 0; c < kPieces; ++c) {
+            const size_t row0 = (size_t)((long long)n_groups * c / kPieces) * N;
+            const size_t row1 = (size_t)((long long)n_groups * (c + 1) / kPieces) * N;
+            const long long s0 = row_start[row0], s1 = row_start[row1];
+            if (s1 > s0)
+                SR_CUDA_TRY(cudaMemcpyAsync(d_packed + s0, symbols + s0, (size_t)(s1 - s0) * 4,
+                                            cudaMemcpyHostToDevice, cs));
+            SR_CUDA_TRY(cudaEventCreateWithFlags(&copied[c], cudaEventDisableTiming));
+            SR_CUDA_TRY(cudaEventRecord(copied[c], cs));
+        }
+        f.copied = copied;
+        f.pieces = kPieces;
+        const GroupFeed feed{kPieces, feed_piece, &f};
+        const int rc = launch_gate_multi(ga, di + h.off_ws, h.total - h.off_ws, s, nullptr, false, nullptr, &feed);
+        for (int c = 0; c < kPieces; ++c) cudaEventDestroy(copied[c]);   // released once completed
+        if (rc != SR_OK) return rc;
+    } else {
+        SR_CUDA_TRY(cudaMemcpyAsync(d_start, row_start, (rows + 1) * 8, cudaMemcpyHostToDevice, s));
+        if (total > 0)
+            SR_CUDA_TRY(cudaMemcpyAsync(d_packed, symbols, (size_t)total * 4, cudaMemcpyHostToDevice, s));
+        int rc = unpack_rows(f, 0, n_groups, s);
+        if (rc != SR_OK) return rc;
+        rc = sr_gate(ga.seqs, ga.lens, n_groups, N, stride, K, threshold, norm_mode, ga.pair_dist,
+                     ga.pair_sum, ga.mean, ga.stop, ga.status, di + h.off_ws, h.total - h.off_ws, stream);
+        if (rc != SR_OK) return rc;
+    }
     if (pair_dist)
         SR_CUDA_TRY(cudaMemcpyAsync(pair_dist, di + h.off_dist, (size_t)n_groups * P * 4,
                                     cudaMemcpyDeviceToHost, s));

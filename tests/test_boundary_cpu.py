@@ -164,7 +164,7 @@ def test_packed_host_entry_rejects_bad_offsets_before_any_launch(lib):
     def call(row_start, stride=32, K=30, n_groups=1, N=2):
         rs = np.asarray(row_start, dtype=np.int64)
         return fn(sym.ctypes.data, rs.ctypes.data, n_groups, N, stride, K, 0.5, 0, None, None, None,
-                  stop.ctypes.data, None, None, 0, None)
+                  stop.ctypes.data, None, None, 0, None, None)
 
     assert call([1, 5, 9]) == binding.SR_ERR_BAD_OFFSETS          # does not begin at 0
     assert call([0, 9, 5]) == binding.SR_ERR_BAD_OFFSETS          # decreases

@@ -234,9 +234,10 @@ def _check_stream(s, G=None):
 
 def test_packed_host_entry_point():
     """Packed (ragged) host input: same outputs as the oracle on the padded batch, on the
-    single-word and the multi-word path, with empty rows and rows longer than K, twice in
-    a row on one arena."""
+    single-word and the multi-word path, with empty rows and rows longer than K, in one
+    piece and in pieces on a copy stream, on one arena."""
     dev = torch.device("cuda:0")
+    cs = torch.cuda.Stream(device=dev)
     cases = [(W.agent_gate(K=15), 15), (W.token_gate(n_groups=72), 1024), (W.token_gate(n_groups=72), 500)]
     for w, K in cases:
         lens = w.lens.copy()
@@ -248,17 +249,17 @@ def test_packed_host_entry_point():
         h_sym = torch.from_numpy(symbols).pin_memory()
         h_rs = torch.from_numpy(row_start).pin_memory()
         arena = torch.empty(sr.sr_gate_host_packed_arena_bytes(G, N, stride, K), dtype=torch.uint8, device=dev)
-        for rep in range(2):
+        for copy_stream in (None, cs, cs):
             pd = torch.full((G, P), -7, dtype=torch.int32).pin_memory()
             ps = torch.full((G,), -7, dtype=torch.int32).pin_memory()
             mean = torch.full((G,), -7.0, dtype=torch.float64).pin_memory()
             stop = torch.full((G,), 9, dtype=torch.uint8).pin_memory()
             st = torch.zeros(1, dtype=torch.int32).pin_memory()
             sr.sr_gate_host_packed(h_sym, h_rs, N, stride, K, 0.3, w.norm_mode, pair_dist=pd, pair_sum=ps,
-                                   mean=mean, stop=stop, status=st, arena=arena)
+                                   mean=mean, stop=stop, status=st, arena=arena, copy_stream=copy_stream)
             torch.cuda.synchronize()
             assert_gate_matches((pd.numpy(), ps.numpy(), mean.numpy(), stop.numpy()), want,
-                                f"packed {w.name} K={K} call {rep}")
+                                f"packed {w.name} K={K} copy stream {copy_stream is not None}")
             assert int(st.item()) == 0
 
 
