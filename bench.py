@@ -327,7 +327,7 @@ def main():
                 "ms_per_step": e2e_ms / args.steps,
                 "input": "packed prefixes + int64 row offsets in pinned host memory (sr_gate_host_packed), "
                          "sent in four pieces on a copy stream under the per-group pass; one recurrence launch"},
-        "gpu_launches": 6 * args.steps,
+        "gpu_launches": 5 * args.steps,
         "clocks": clocks,
         "stage_ms": {"prep": stage_ms[0], "order": stage_ms[1], "dp": stage_ms[2], "finish": stage_ms[3]},
         "roofline": {"kernel": "multi_dp_kernel", "bound": "alu", "achieved": achieved, "peak": alu_peak,

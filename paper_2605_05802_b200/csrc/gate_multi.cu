@@ -5,7 +5,7 @@
 // block keeps its +1 / -1 vertical deltas in two 32-bit words and is advanced one
 // text column at a time by the bit-vector recurrence, with the horizontal delta
 // leaving a block entering the block below.  The work is organised as a pipeline
-// of five launches on the caller's stream, sharing a caller-provided workspace:
+// of four launches on the caller's stream, sharing a caller-provided workspace:
 //
 //   prep     one CTA per (group, pattern rollout): hashes the pattern's symbols
 //            in shared memory, then translates every text paired with it into a
@@ -14,9 +14,8 @@
 //            the pattern's chain).  A block's match word is then just
 //            1 << (loc - first_row_of_block), no table lookup.  Also bins the pairs
 //            by (team shape, text length).
-//   scan     one CTA: prefix sums of the bins, warp-task table.
-//   scatter  orders the pairs: longest warp tasks first, one team shape and similar
-//            text lengths per bin.
+//   order    counting sort of the pairs by bin: longest warp tasks first, one team
+//            shape and similar text lengths per bin; warp-task table.
 //   dp       persistent warps pull tasks.  A task is a warp of 32/T teams; a team of
 //            T lanes (T in {1, 2, 4, 8}) owns one pair, lane l holding R <= 8 consecutive
 //            blocks (32*R rows) in registers.  Lanes are skewed by four columns; the
@@ -310,53 +309,66 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
     if (neg && tid == 0 && a.status) atomicOr(a.status, SR_STATUS_NEG_LEN);
 }
 
-// ------------------------------------------------------------------------ scan
-__global__ void __launch_bounds__(kNumBins)
-multi_scan_kernel(Ctl* ctl) {
-    __shared__ int32_t s[kNumBins];
-    const int t = threadIdx.x;
-    const int own = ctl->hist[t];
-    s[t] = own;
-    __syncthreads();
-    for (int d = 1; d < kNumBins; d <<= 1) {
-        const int v = t >= d ? s[t - d] : 0;
-        __syncthreads();
-        s[t] += v;
-        __syncthreads();
+// ----------------------------------------------------------------------- order
+// Exclusive prefix sum over the kNumBins threads of a CTA (one value per thread).
+__device__ __forceinline__ int block_exclusive_scan(int v, int* s_part /* [32] */) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += up;
     }
-    ctl->start[t] = s[t] - own;
-    ctl->fill[t] = 0;
-    ctl->hist[t] = 0;                  // ready for the next call on this workspace
-    // warp tasks per bin (32 / T pairs per task), exclusive prefix over the bins
-    const int tpw = 32 >> ((t % kNumClasses) / kMaxR);
-    const int own_tasks = (own + tpw - 1) / tpw;
+    if (lane == 31) s_part[warp] = incl;
     __syncthreads();
-    s[t] = own_tasks;
+    if (warp == 0) {
+        const int w = s_part[lane];
+        int wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int up = __shfl_up_sync(0xFFFFFFFFu, wi, d);
+            if (lane >= d) wi += up;
+        }
+        s_part[lane] = wi - w;
+    }
     __syncthreads();
-    for (int d = 1; d < kNumBins; d <<= 1) {
-        const int v = t >= d ? s[t - d] : 0;
-        __syncthreads();
-        s[t] += v;
-        __syncthreads();
-    }
-    ctl->task_start[t] = s[t] - own_tasks;
-    if (t == kNumBins - 1) {
-        ctl->task_start[kNumBins] = s[t];
-        ctl->total_tasks = s[t];
-        ctl->task_counter = 0;
-    }
+    const int r = incl - v + s_part[warp];
+    __syncthreads();                       // s_part may be reused at once
+    return r;
 }
 
-// --------------------------------------------------------------------- scatter
-__global__ void __launch_bounds__(256)
-multi_scatter_kernel(const PairDesc* descs, int32_t* order, Ctl* ctl, int n_pairs) {
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+// Counting sort of the pairs by bin: longest warp tasks first, one team shape and similar
+// text lengths per bin.  Every CTA turns the bin counts into bin starts by itself (a scan
+// of kNumBins values costs less than a launch) and places kNumBins pairs; the first CTA
+// also leaves the tables the dp kernel reads.  `fill` is zeroed by the caller's memset.
+__global__ void __launch_bounds__(kNumBins)
+multi_order_kernel(const PairDesc* descs, int32_t* order, Ctl* ctl, int n_pairs) {
+    __shared__ int s_part[32];
+    __shared__ int32_t s_start[kNumBins];
+    const int t = threadIdx.x;
+    const int own = ctl->hist[t];
+    const int start = block_exclusive_scan(own, s_part);
+    s_start[t] = start;
+    if (blockIdx.x == 0) {
+        // warp tasks per bin (32 / T pairs per task), exclusive prefix over the bins
+        const int tpw = 32 >> ((t % kNumClasses) / kMaxR);
+        const int own_tasks = (own + tpw - 1) / tpw;
+        const int task_start = block_exclusive_scan(own_tasks, s_part);
+        ctl->start[t] = start;
+        ctl->task_start[t] = task_start;
+        if (t == kNumBins - 1) {
+            ctl->task_start[kNumBins] = task_start + own_tasks;
+            ctl->total_tasks = task_start + own_tasks;
+            ctl->task_counter = 0;
+        }
+    }
+    __syncthreads();
+    const int idx = blockIdx.x * kNumBins + t;
     if (idx >= n_pairs) return;
     const uint32_t b = descs[idx].bin;
     if (!(b & kNeedsDp)) return;
     const int bin = (int)(b & kBinMask);
-    const int pos = ctl->start[bin] + atomicAdd(&ctl->fill[bin], 1);
-    order[pos] = idx;
+    order[s_start[bin] + atomicAdd(&ctl->fill[bin], 1)] = idx;
 }
 
 // -------------------------------------------------------------------------- dp
@@ -653,7 +665,9 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     const int prep_smem = hslots * 8 + W.pitch * 4;
 
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[0], s));
-    SR_CUDA_TRY(cudaMemsetAsync(ctl->hist, 0, sizeof(ctl->hist), s));
+    // bin counts (filled by prep) and fill counters (used by the ordering kernel) start at zero
+    static_assert(offsetof(Ctl, fill) + sizeof(Ctl::fill) == 3 * kNumBins * sizeof(int32_t), "hist, start, fill lead Ctl");
+    SR_CUDA_TRY(cudaMemsetAsync(ctl, 0, 3 * kNumBins * sizeof(int32_t), s));
     uint8_t* flag = decide ? ws + W.off_flag : nullptr;
     // The match-stream pass works group by group, so when the groups arrive in pieces it runs
     // piece by piece: `feed->before` enqueues whatever makes groups [g0, g1) ready on `s`.
@@ -678,12 +692,10 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
         SR_LAUNCH_CHECK("multi_bound_kernel");
     }
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[1], s));
-    multi_scan_kernel<<<1, kNumBins, 0, s>>>(ctl);
-    SR_LAUNCH_CHECK("multi_scan_kernel");
-    multi_scatter_kernel<<<(n_pairs + 255) / 256, 256, 0, s>>>(
+    multi_order_kernel<<<(n_pairs + kNumBins - 1) / kNumBins, kNumBins, 0, s>>>(
         reinterpret_cast<const PairDesc*>(ws + W.off_desc),
         reinterpret_cast<int32_t*>(ws + W.off_order), ctl, n_pairs);
-    SR_LAUNCH_CHECK("multi_scatter_kernel");
+    SR_LAUNCH_CHECK("multi_order_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[2], s));
     int dev = 0, sms = 0;
     SR_CUDA_TRY(cudaGetDevice(&dev));
