@@ -472,6 +472,12 @@ def main():
                                        "gcups": W.dp_cells(w0.lens, K) / (all0 * 1e-3) / 1e9,
                                        "word_columns": wc0, "dp_alu_gops": 10.0 * wc0 / (dp0 * 1e-3) / 1e9,
                                        "dp_alu_frac": 10.0 * wc0 / (dp0 * 1e-3) / 1e9 / alu_peak}
+        # small token-level batches (teams of up to a whole warp per pair)
+        for small in (16, 64):
+            ws_ = W.token_gate(seed=3, n_groups=small)
+            r_ = gate_case(ws_)
+            r_.pop("alu_gops"), r_.pop("alu_frac")        # those two count single-word columns
+            extras[f"C4_{small}_groups"] = r_
         # a large batch of action-level groups at the paper's G = 8, K = 15
         extras["C2_x128_groups"] = gate_case(W.agent_gate(K=15, n_groups=65536), reps=10)
         # the rows beyond the gate proper: OR rule, Appendix-B signals, batch statistics

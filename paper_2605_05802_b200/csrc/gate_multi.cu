@@ -17,7 +17,7 @@
 //   order    counting sort of the pairs by bin: longest warp tasks first, one team
 //            shape and similar text lengths per bin; warp-task table.
 //   dp       persistent warps pull tasks.  A task is a warp of 32/T teams; a team of
-//            T lanes (T in {1, 2, 4, 8}) owns one pair, lane l holding R <= 8 consecutive
+//            T lanes (T in {1, 2, 4, 8}; up to 32 in small batches) owns one pair, lane l holding R <= 6 consecutive
 //            blocks (32*R rows) in registers.  Lanes are skewed by four columns; the
 //            delta words of a lane's last block reach the next lane by warp shuffles.
 //            All pairs of a task share (T, R) and have similar lengths, so the warp's
@@ -34,7 +34,7 @@ namespace {
 
 constexpr int kPrepThreads = 256;
 constexpr int kMaxR = 8;            // blocks (32 rows each) per lane
-constexpr int kNumClasses = 32;     // class = log2(T) * kMaxR + (R - 1), T in {1, 2, 4, 8}
+constexpr int kNumClasses = 32;     // team shapes (T lanes x R blocks), see class_of
 constexpr int kLenBuckets = 32;     // buckets of estimated task duration
 constexpr int kNumBins = kNumClasses * kLenBuckets;
 constexpr uint32_t kLocNone = 0x7FFFu;    // bit 15 clear, far above any row: shifts to 0
@@ -66,12 +66,14 @@ struct Ctl {               // int32 control block in the workspace
 struct MultiWs {
     size_t off_dist, off_desc, off_loc, off_next, off_order, off_ctl, off_flag, total;
     int pitch;             // uint16 elements per loc / chain row
+    int min_tlog;          // small batches: teams of at least 2^min_tlog lanes
 };
 
 MultiWs multi_layout(int32_t n_groups, int32_t N, int32_t K) {
     MultiWs w;
     const size_t P = pairs_of(N);
     w.pitch = (K + 7) & ~7;
+    w.min_tlog = 0;
     size_t off = 0;
     w.off_ctl = off;   off = align_up(off + sizeof(Ctl), 256);
     w.off_flag = off;  off = align_up(off + (size_t)n_groups, 256);
@@ -84,7 +86,7 @@ MultiWs multi_layout(int32_t n_groups, int32_t N, int32_t K) {
     return w;
 }
 
-__host__ __device__ inline void team_shape(int m, int& tlog, int& R) {
+__host__ __device__ inline void team_shape(int m, int min_tlog, int& tlog, int& R) {
     // T lanes x R blocks per lane >= W blocks of the pattern, with little padding and
     // R large enough to amortise the per-column work that does not depend on R
     const int W = (m + 31) >> 5;            // <= 32
@@ -92,6 +94,28 @@ __host__ __device__ inline void team_shape(int m, int& tlog, int& R) {
     else if (W <= 12) { tlog = 1; R = (W + 1) >> 1; }
     else if (W <= 24) { tlog = 2; R = (W + 3) >> 2; }
     else { tlog = 3; R = (W + 7) >> 3; }
+    // A batch with too few pairs to give every resident warp its tasks spreads a pair over
+    // more lanes (up to the whole warp): shorter tasks, more of them.
+    if (tlog < min_tlog) {
+        int t = tlog;
+        while (t < min_tlog && (1 << t) < W) ++t;
+        tlog = t;
+        R = (W + (1 << t) - 1) >> t;
+    }
+}
+
+// Class of a team shape.  T = 1, 2, 4, 8 with R = 1..6 fill slots log2(T) * 8 + R - 1; the
+// shapes of small batches, T = 16 with R = 1, 2 and T = 32 with R = 1, take slots 6, 7, 14.
+__host__ __device__ inline int class_of(int tlog, int R) {
+    if (tlog < 4) return tlog * 8 + (R - 1);
+    return tlog == 4 ? 5 + R : 14;
+}
+__host__ __device__ inline void shape_of_class(int cls, int& tlog, int& R) {
+    if ((cls & 7) < 6) { tlog = cls >> 3; R = (cls & 7) + 1; }
+    else if (cls == 6) { tlog = 4; R = 1; }
+    else if (cls == 7) { tlog = 4; R = 2; }
+    else if (cls == 14) { tlog = 5; R = 1; }
+    else { tlog = 0; R = 1; }               // unused slots: no pair ever lands here
 }
 
 // Bins order the pairs by the estimated running time of their warp task (text
@@ -104,7 +128,7 @@ __host__ __device__ inline int bin_of(int n, int tlog, int R) {
     const int max_cost = (SR_MAX_K + 32) * (14 * kMaxR + 20) + 1;
     int bucket = (int)(((long long)cost * kLenBuckets) / max_cost);
     bucket = bucket < 0 ? 0 : (bucket >= kLenBuckets ? kLenBuckets - 1 : bucket);
-    return (kLenBuckets - 1 - bucket) * kNumClasses + (tlog * kMaxR + (R - 1));
+    return (kLenBuckets - 1 - bucket) * kNumClasses + class_of(tlog, R);
 }
 
 __device__ __forceinline__ int clamp_len(const int32_t* lens, size_t idx, int K, bool& neg) {
@@ -297,7 +321,7 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
                                   (uint32_t)abs(m - n)};
         } else {
             int tlog, R;
-            team_shape(m - strip, tlog, R);
+            team_shape(m - strip, W.min_tlog, tlog, R);
             const int bin = bin_of(n - strip, tlog, R);
             const int lower = kBounds ? max(abs(m - n), s_absent[tid]) : 0;
             descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i),
@@ -351,7 +375,9 @@ multi_order_kernel(const PairDesc* descs, int32_t* order, Ctl* ctl, int n_pairs)
     s_start[t] = start;
     if (blockIdx.x == 0) {
         // warp tasks per bin (32 / T pairs per task), exclusive prefix over the bins
-        const int tpw = 32 >> ((t % kNumClasses) / kMaxR);
+        int tl, rr;
+        shape_of_class(t % kNumClasses, tl, rr);
+        const int tpw = 32 >> tl;
         const int own_tasks = (own + tpw - 1) / tpw;
         const int task_start = block_exclusive_scan(own_tasks, s_part);
         ctl->start[t] = start;
@@ -522,8 +548,8 @@ multi_dp_kernel(unsigned char* ws, MultiWs W, int32_t* dist_out, uint32_t two) {
             const int mid = (k + hi) >> 1;
             if (ctl->task_start[mid] <= task) k = mid; else hi = mid;
         }
-        const int cls = k % kNumClasses;
-        const int tlog = cls / kMaxR, R = cls % kMaxR + 1;
+        int tlog, R;
+        shape_of_class(k % kNumClasses, tlog, R);
         const int tpw = 32 >> tlog;
         const int pos = ctl->start[k] + (task - ctl->task_start[k]) * tpw + (lane >> tlog);
         const bool valid = pos < ctl->start[k] + ctl->fill[k];     // fill = pairs in the bin
@@ -533,9 +559,7 @@ multi_dp_kernel(unsigned char* ws, MultiWs W, int32_t* dist_out, uint32_t two) {
             case 3: dp_task<3>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
             case 4: dp_task<4>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
             case 5: dp_task<5>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
-            case 6: dp_task<6>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
-            case 7: dp_task<7>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
-            default: dp_task<8>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+            default: dp_task<6>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
         }
     }
 }
@@ -649,13 +673,22 @@ size_t gate_multi_workspace_bytes(int32_t n_groups, int32_t N, int32_t stride, i
 int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_t s,
                       const cudaEvent_t* ev, bool decide, uint8_t* exact, const GroupFeed* feed) {
     if (a.n_groups == 0) return SR_OK;
-    const MultiWs W = multi_layout(a.n_groups, a.N, a.K);
+    MultiWs W = multi_layout(a.n_groups, a.N, a.K);
     if (ws_ == nullptr || ws_bytes < W.total || (reinterpret_cast<uintptr_t>(ws_) & 255) != 0)
         return SR_ERR_WORKSPACE;
     unsigned char* ws = static_cast<unsigned char*>(ws_);
     const int P = pairs_of(a.N);
     const long long n_pairs_ll = (long long)a.n_groups * P;
     if (n_pairs_ll > 0x7FFFFFFFLL) return SR_ERR_BAD_N;
+    int dev = 0, sms = 0;
+    SR_CUDA_TRY(cudaGetDevice(&dev));
+    SR_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    // fewer than two pairs per resident warp (12 warps per SM): widen the teams until there
+    // are about eight lanes' worth of pairs per warp (measured on token-level batches of 16 to
+    // 256 groups: -40 % at 16 groups, -22 % at 64, nothing to gain from 128 on)
+    const long long warps = 12LL * sms;
+    if (n_pairs_ll < 2 * warps)
+        while (W.min_tlog < 5 && (n_pairs_ll << W.min_tlog) < 8 * warps) ++W.min_tlog;
     const int n_pairs = (int)n_pairs_ll;
     int32_t* dist = a.pair_dist ? a.pair_dist : reinterpret_cast<int32_t*>(ws + W.off_dist);
     Ctl* ctl = reinterpret_cast<Ctl*>(ws + W.off_ctl);
@@ -697,9 +730,6 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
         reinterpret_cast<int32_t*>(ws + W.off_order), ctl, n_pairs);
     SR_LAUNCH_CHECK("multi_order_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[2], s));
-    int dev = 0, sms = 0;
-    SR_CUDA_TRY(cudaGetDevice(&dev));
-    SR_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     // persistent grid: a multiple of the SM count; warps pull tasks until none is left
     long long want = (n_pairs_ll + kDpWarpsPerCta - 1) / kDpWarpsPerCta;
     // 3 CTAs of 4 warps per SM (3 warps per scheduler): enough to keep the integer pipe

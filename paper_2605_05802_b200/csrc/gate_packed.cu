@@ -58,6 +58,19 @@ int feed_piece(void* ctx, int g0, int g1, cudaStream_t s) {
     return unpack_rows(f, g0, g1, s);
 }
 
+// Events of one call; destroyed when the call returns, whichever way (an event that is
+// still pending is released by the driver once it has completed).
+struct EventSet {
+    cudaEvent_t ev[8];
+    int n = 0;
+    cudaError_t add() {
+        const cudaError_t e = cudaEventCreateWithFlags(&ev[n], cudaEventDisableTiming);
+        if (e == cudaSuccess) ++n;
+        return e;
+    }
+    ~EventSet() { for (int k = 0; k < n; ++k) cudaEventDestroy(ev[k]); }
+};
+
 struct PackedArena {
     size_t off_packed, off_start, inner, total;     // `inner`: where the padded-input arena begins
 };
@@ -135,13 +148,11 @@ int sr_gate_host_packed(const int32_t* symbols, const int64_t* row_start, int32_
     // time of the recurrence launch.
     if (cs != nullptr && cs != s && K > 32 && n_groups >= 64) {
         constexpr int kPieces = 4;
-        cudaEvent_t copied[kPieces];
-        cudaEvent_t ev = nullptr;
+        EventSet events;                                  // [0] fork, [1 + c] piece c copied
+        for (int k = 0; k < 1 + kPieces; ++k) SR_CUDA_TRY(events.add());
         // the copies must not overtake earlier work on `stream` that uses the arena
-        SR_CUDA_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
-        SR_CUDA_TRY(cudaEventRecord(ev, s));
-        SR_CUDA_TRY(cudaStreamWaitEvent(cs, ev, 0));
-        SR_CUDA_TRY(cudaEventDestroy(ev));               // released once it has completed
+        SR_CUDA_TRY(cudaEventRecord(events.ev[0], s));
+        SR_CUDA_TRY(cudaStreamWaitEvent(cs, events.ev[0], 0));
         SR_CUDA_TRY(cudaMemcpyAsync(d_start, row_start, (rows + 1) * 8, cudaMemcpyHostToDevice, cs));
         for (int c = 0; c < kPieces; ++c) {
             const size_t row0 = (size_t)((long long)n_groups * c / kPieces) * N;
@@ -150,14 +161,12 @@ int sr_gate_host_packed(const int32_t* symbols, const int64_t* row_start, int32_
             if (s1 > s0)
                 SR_CUDA_TRY(cudaMemcpyAsync(d_packed + s0, symbols + s0, (size_t)(s1 - s0) * 4,
                                             cudaMemcpyHostToDevice, cs));
-            SR_CUDA_TRY(cudaEventCreateWithFlags(&copied[c], cudaEventDisableTiming));
-            SR_CUDA_TRY(cudaEventRecord(copied[c], cs));
+            SR_CUDA_TRY(cudaEventRecord(events.ev[1 + c], cs));
         }
-        f.copied = copied;
+        f.copied = events.ev + 1;
         f.pieces = kPieces;
         const GroupFeed feed{kPieces, feed_piece, &f};
         const int rc = launch_gate_multi(ga, di + h.off_ws, h.total - h.off_ws, s, nullptr, false, nullptr, &feed);
-        for (int c = 0; c < kPieces; ++c) cudaEventDestroy(copied[c]);   // released once completed
         if (rc != SR_OK) return rc;
     } else {
         SR_CUDA_TRY(cudaMemcpyAsync(d_start, row_start, (rows + 1) * 8, cudaMemcpyHostToDevice, s));

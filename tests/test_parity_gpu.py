@@ -103,6 +103,16 @@ def test_multiword_maximum_sizes_and_degenerate_groups():
     assert_gate_matches(got, want, "one symbol")
 
 
+@pytest.mark.parametrize("n_groups", [1, 8, 40, 100, 130])
+def test_multiword_small_batches(n_groups):
+    """Small token-level batches: the multi-word path spreads a pair over more lanes (up to a
+    whole warp) when there are too few pairs to fill the machine; same outputs at every size."""
+    w = W.token_gate(seed=11, n_groups=n_groups, min_len=40, max_len=1024)
+    want = oracle.gate(w.seqs, w.lens, w.K, 0.4, w.norm_mode, threads=8)
+    got = gate_gpu(w.seqs, w.lens, w.K, 0.4, w.norm_mode)
+    assert_gate_matches(got, want, f"{n_groups} groups")
+
+
 def test_multiword_shared_prefixes():
     """Rollouts that agree on their first symbols: the multi-word path leaves the common
     prefix of a pair out of the recurrence, so every prefix length around its 4-symbol
