@@ -53,6 +53,7 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
     __shared__ uint32_t s_bits[SR_MAX_N * kBgWords];
     __shared__ int s_nbig;
     __shared__ double s_term[SR_MAX_N * (SR_MAX_N - 1) / 2];
+    __shared__ double s_plogp[SR_MAX_N];
     const int g = blockIdx.x, tid = threadIdx.x, nthr = blockDim.x;
     const int P = pairs_of(N);
     for (int i = tid; i < N; i += nthr) {
@@ -133,6 +134,11 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
             s_term[p] = uni > 0 ? __dsub_rn(1.0, __ddiv_rn((double)both, (double)uni)) : 0.0;
         }
     }
+    // entropy terms side by side (the logarithms are the long part); added up in order below
+    if (tid < N) {
+        const double pr = __ddiv_rn((double)s_same[tid], (double)N);
+        s_plogp[tid] = s_fa[tid] ? __dmul_rn(pr, log(pr)) : 0.0;
+    }
     __syncthreads();
     if (tid == 0) {
         int dp = 0, da = 0;
@@ -140,10 +146,7 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
         for (int i = 0; i < N; ++i) {
             dp += s_fp[i];
             da += s_fa[i];
-            if (s_fa[i]) {
-                const double pr = __ddiv_rn((double)s_same[i], (double)N);
-                h = __dsub_rn(h, __dmul_rn(pr, log(pr)));
-            }
+            if (s_fa[i]) h = __dsub_rn(h, s_plogp[i]);
         }
         if (upr) upr[g] = __ddiv_rn((double)dp, (double)N);
         if (uar) uar[g] = __ddiv_rn((double)da, (double)N);
