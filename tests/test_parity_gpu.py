@@ -103,6 +103,31 @@ def test_multiword_maximum_sizes_and_degenerate_groups():
     assert_gate_matches(got, want, "one symbol")
 
 
+def test_multiword_null_lengths_raw_norm_and_negative_lengths():
+    """The multi-word path with lens = NULL (every prefix has K symbols), with the raw-distance
+    normalisation, and with negative lengths (treated as 0 and flagged)."""
+    rng = np.random.default_rng(41)
+    G, N, stride = 7, 6, 104
+    seqs = rng.integers(0, 30, size=(G, N, stride)).astype(np.int32)
+    for K in (100, 33):
+        full = np.full((G, N), K, dtype=np.int32)
+        want = oracle.gate(seqs, full, K, 0.8)
+        got = gate_gpu(seqs, None, K, 0.8)
+        assert_gate_matches(got, want, f"lens=NULL K={K}")
+    lens = rng.integers(40, 101, size=(G, N)).astype(np.int32)
+    want = oracle.gate(seqs, lens, 100, 70.0, sr.SR_NORM_NONE)
+    got = gate_gpu(seqs, lens, 100, 70.0, sr.SR_NORM_NONE)
+    assert_gate_matches(got, want, "raw distances")
+    assert 0 < want[3].sum() < G
+    lens[2, 3] = -5
+    lens[4, 0] = -1
+    status = []
+    want = oracle.gate(seqs, np.maximum(lens, 0), 100, 0.8)
+    got = gate_gpu(seqs, lens, 100, 0.8, status=status)
+    assert_gate_matches(got, want, "negative lengths")
+    assert status[0] & sr.SR_STATUS_NEG_LEN
+
+
 @pytest.mark.parametrize("n_groups", [1, 8, 40, 100, 130])
 def test_multiword_small_batches(n_groups):
     """Small token-level batches: the multi-word path spreads a pair over more lanes (up to a
