@@ -328,6 +328,27 @@ int sr_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_groups,
 int sr_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int32_t N,
                    int64_t* counts, double* sumsq, void* stream);
 
+/*
+ * sr_kept_groups -- the groups that stay in the training batch, as an index list.  The
+ * trainer skips a group the gate cut (Appendix C.1); the dynamic-sampling baseline the
+ * paper compares with (appendix on strong baselines) also drops the groups whose
+ * advantages are all zero (Section 2.1).  This call writes the ascending indices g of the
+ * groups with stop[g] == 0 and, when zero_var is given, zero_var[g] == 0.
+ *
+ *   stop       in  [n_groups] uint8 or NULL (no group cut)
+ *   zero_var   in  [n_groups] uint8 or NULL (filter off)
+ *   index      out [n_groups] int32; the first *count entries are written, ascending
+ *   count      out 1 int32 (device)
+ *   workspace      device scratch of sr_kept_groups_workspace_bytes(n_groups) bytes,
+ *                  16-byte aligned; contents undefined before and after
+ *
+ * The order does not depend on how the kernels are scheduled.  n_groups == 0 writes
+ * *count = 0.
+ */
+int sr_kept_groups(const uint8_t* stop, const uint8_t* zero_var, int32_t n_groups, int32_t* index,
+                   int32_t* count, void* workspace, size_t workspace_bytes, void* stream);
+size_t sr_kept_groups_workspace_bytes(int32_t n_groups);   /* host-only, pure */
+
 /* Host-only, pure.  Step-token saving of cutting `cut` of `n_groups` groups at step K of
  * a horizon of T_max steps: cut * (T_max - K) / (n_groups * T_max) (caption of Table 1). */
 double sr_savings_fraction(int64_t cut, int64_t n_groups, int32_t T_max, int32_t K);

@@ -70,6 +70,8 @@ def _load():
         lib.sro_group_signals.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                           ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_void_p, ctypes.c_void_p]
+        lib.sro_kept_groups.restype = ctypes.c_int32
+        lib.sro_kept_groups.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]
         lib.sro_max_threads.restype = ctypes.c_int32
         _lib = lib
     return _lib
@@ -187,6 +189,22 @@ def batch_stats(adv: np.ndarray, stop: Optional[np.ndarray]):
     sumsq = np.zeros(2, dtype=np.float64)
     _load().sro_batch_stats(adv.ctypes.data, sp, G, N, counts.ctypes.data, sumsq.ctypes.data)
     return counts, sumsq
+
+
+def kept_groups(stop: Optional[np.ndarray], zero_var: Optional[np.ndarray] = None,
+                n_groups: Optional[int] = None) -> np.ndarray:
+    """Ascending indices (int32) of the groups that stay in the batch: not cut
+    (Appendix C.1) and, when ``zero_var`` is given, not zero-variance either."""
+    sp = zp = None
+    if stop is not None:
+        stop = np.ascontiguousarray(stop, dtype=np.uint8)
+        sp, n_groups = stop.ctypes.data, stop.shape[0]
+    if zero_var is not None:
+        zero_var = np.ascontiguousarray(zero_var, dtype=np.uint8)
+        zp, n_groups = zero_var.ctypes.data, zero_var.shape[0]
+    index = np.zeros(max(int(n_groups), 1), dtype=np.int32)
+    kept = int(_load().sro_kept_groups(sp, zp, int(n_groups), index.ctypes.data))
+    return index[:kept].copy()
 
 
 def savings_fraction(cut: int, n_groups: int, T_max: int, K: int) -> float:

@@ -279,6 +279,22 @@ void sro_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, in
     }
 }
 
+/* Groups that stay in the training batch, ascending: a cut group is skipped by the
+ * trainer (Appendix C.1), and with the zero-variance filter of the dynamic-sampling
+ * baseline (Appendix on strong baselines) so is a group whose advantages are all zero
+ * (Section 2.1).  Returns how many indices were written to `index`. */
+int32_t sro_kept_groups(const uint8_t* stop, const uint8_t* zero_var, int32_t n_groups,
+                        int32_t* index) {
+    int32_t kept = 0;
+    for (int32_t g = 0; g < n_groups; ++g) {
+        if (stop && stop[g] != 0) continue;
+        if (zero_var && zero_var[g] != 0) continue;
+        index[kept] = g;
+        kept = kept + 1;
+    }
+    return kept;
+}
+
 /* Step-token saving of cutting `cut` of `n_groups` groups at step K of T_max
  * (caption of Table 1): cut * (T_max - K) / (n_groups * T_max). */
 double sro_savings_fraction(int64_t cut, int64_t n_groups, int32_t T_max, int32_t K) {

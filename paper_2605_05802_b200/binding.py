@@ -54,6 +54,8 @@ _SIGNATURES = {
     "sr_gate_or_rule": (ctypes.c_int, [_vp, _vp, _vp, _i32, _i32, _i32, _f64, _f64, _vp, _vp, _vp]),
     "sr_group_signals": (ctypes.c_int, [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "sr_batch_stats": (ctypes.c_int, [_vp, _vp, _i32, _i32, _vp, _vp, _vp]),
+    "sr_kept_groups": (ctypes.c_int, [_vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp]),
+    "sr_kept_groups_workspace_bytes": (_sz, [_i32]),
     "sr_savings_fraction": (ctypes.c_double, [ctypes.c_int64, ctypes.c_int64, _i32, _i32]),
     "sr_dilution_gain": (ctypes.c_double, [_f64, _f64]),
     "sr_grpo_advantage": (ctypes.c_int, [_vp, _vp, _i32, _i32, _f32, _vp, _vp, _vp]),
@@ -279,6 +281,23 @@ def sr_batch_stats(adv: torch.Tensor, stop: Optional[torch.Tensor], *, counts: t
     G, N = adv.shape
     _check(load().sr_batch_stats(_ptr(adv, torch.float32), _ptr(stop, torch.uint8), G, N,
                                  _ptr(counts, torch.int64), _ptr(sumsq, torch.float64), _stream(stream)))
+
+
+def sr_kept_groups_workspace_bytes(n_groups: int) -> int:
+    return int(load().sr_kept_groups_workspace_bytes(n_groups))
+
+
+def sr_kept_groups(stop: Optional[torch.Tensor], zero_var: Optional[torch.Tensor], *, index: torch.Tensor,
+                   count: torch.Tensor, workspace: Optional[torch.Tensor], n_groups: Optional[int] = None,
+                   stream=None) -> None:
+    """index int32 [n_groups], count int32 [1] (device): ascending indices of the groups
+    with stop == 0 (and zero_var == 0 when given)."""
+    if n_groups is None:
+        n_groups = (stop if stop is not None else zero_var if zero_var is not None else index).shape[0]
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().sr_kept_groups(_ptr(stop, torch.uint8), _ptr(zero_var, torch.uint8), n_groups,
+                                 _ptr(index, torch.int32), _ptr(count, torch.int32), _ptr(workspace),
+                                 ws_bytes, _stream(stream)))
 
 
 def sr_savings_fraction(cut: int, n_groups: int, T_max: int, K: int) -> float:

@@ -13,7 +13,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsr_gate.so")
 SOURCES = ["api.cu", "gate_single.cu", "gate_multi.cu", "incremental.cu", "advantage.cu", "probe.cu",
-           "gate_noalloc.cu", "signals.cu", "gate_packed.cu"]
+           "gate_noalloc.cu", "signals.cu", "gate_packed.cu", "compact.cu"]
 
 
 def _stale() -> bool:

@@ -284,6 +284,22 @@ int sr_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int3
     return launch_batch_stats(adv, stop, n_groups, N, counts, sumsq, static_cast<cudaStream_t>(stream));
 }
 
+size_t sr_kept_groups_workspace_bytes(int32_t n_groups) {
+    if (n_groups < 0) return 0;
+    return kept_groups_workspace_bytes(n_groups);
+}
+
+int sr_kept_groups(const uint8_t* stop, const uint8_t* zero_var, int32_t n_groups, int32_t* index,
+                   int32_t* count, void* workspace, size_t workspace_bytes, void* stream) {
+    if (n_groups < 0) return SR_ERR_BAD_N;
+    if (count == nullptr || (n_groups > 0 && index == nullptr)) return SR_ERR_NULL;
+    if (n_groups > 0 && (workspace == nullptr || workspace_bytes < kept_groups_workspace_bytes(n_groups) ||
+                         (reinterpret_cast<uintptr_t>(workspace) & 15) != 0))
+        return SR_ERR_WORKSPACE;
+    return launch_kept_groups(stop, zero_var, n_groups, index, count, workspace,
+                              static_cast<cudaStream_t>(stream));
+}
+
 double sr_savings_fraction(int64_t cut, int64_t n_groups, int32_t T_max, int32_t K) {
     if (n_groups <= 0 || T_max <= 0) return 0.0;
     return (double)(cut * (int64_t)(T_max - K)) / (double)(n_groups * (int64_t)T_max);

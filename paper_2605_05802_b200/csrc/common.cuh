@@ -121,4 +121,9 @@ int launch_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_gro
 int launch_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, int32_t N,
                        int64_t* counts, double* sumsq, cudaStream_t s);
 
+// compact.cu
+size_t kept_groups_workspace_bytes(int32_t n_groups);
+int launch_kept_groups(const uint8_t* stop, const uint8_t* zero_var, int32_t n_groups,
+                       int32_t* index, int32_t* count, void* ws, cudaStream_t s);
+
 }  // namespace sr
