@@ -11,8 +11,11 @@
  *     allocates no device memory and keeps no state between calls.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls enqueue work on it and return without synchronising.
- *   - Return value: SR_OK, or a negative SR_ERR_* code, in which case nothing was
- *     enqueued and no buffer was touched.
+ *   - Return value: SR_OK, or a negative SR_ERR_* code.  Every code except SR_ERR_CUDA
+ *     comes from a check of the arguments made before anything is enqueued: no buffer
+ *     was touched.  SR_ERR_CUDA reports a CUDA call or launch that failed part-way:
+ *     earlier copies and kernels of the same call may already be on the stream, and the
+ *     outputs, the workspace / arena and *status are then undefined.
  *   - Actions (or tokens) are int32 IDs compared for equality only; every 32-bit
  *     value is legal.  Mapping action strings to IDs is the caller's job.
  *   - Pairs of a group are ordered (0,1),(0,2),...,(0,N-1),(1,2),...,(N-2,N-1);
@@ -197,16 +200,23 @@ size_t sr_gate_host_packed_arena_bytes(int32_t n_groups, int32_t N, int32_t stri
  * call cudaMalloc.  There sr_gate's `workspace` has nowhere to come from.  This
  * entry point takes the same inputs and outputs but no workspace: the multi-word
  * path (K > 32) works in a fixed array of SR_NOALLOC_SCRATCH_BYTES that is part of
- * the library's device image, so every GPU on which the library is used holds that
- * much memory from load until the process exits.  It calls no allocation routine.
+ * the library's device image, so every GPU on which this entry point has been used
+ * holds that much memory until the process exits.  It calls no allocation routine;
+ * the CUDA runtime reserves the array when it loads the image on a device, which with
+ * its default lazy loading happens inside the first call there.
  *
  *   - Limit: sr_gate_workspace_bytes(n_groups, N, stride, K) must not exceed
  *     SR_NOALLOC_SCRATCH_BYTES (also returned by sr_gate_noalloc_limit_bytes());
  *     otherwise SR_ERR_SCRATCH_LIMIT, nothing enqueued.  As a guide, 64 groups of
  *     N = 8 at K = 1024, or 1000 groups at K = 64, fit.  K <= 32 has no limit.
- *   - The first call on each device looks up the array's device address (a
- *     cudaGetSymbolAddress with that device current).  Make that first call during
- *     set-up, before any stream capture is begun.
+ *   - The first call on each device (with K > 32) looks up the array's device address
+ *     (a cudaGetSymbolAddress with that device current), which is also when the 16 MiB
+ *     are reserved.  Make that first call during set-up, before any stream capture is
+ *     begun and while the memory is still to be had: if the device is already full it
+ *     fails with SR_ERR_CUDA.  The address is remembered per device; after a
+ *     cudaDeviceReset it is stale, so do not use this entry point on a device that the
+ *     process has reset.
+ *   - Arguments are checked exactly as sr_gate checks them, before the size limit.
  *   - All calls on a device share the one array.  It keeps whatever the last call
  *     left; each call clears the counters it needs zeroed before using them.  Two
  *     calls that can overlap on the device (different streams, no dependency) race

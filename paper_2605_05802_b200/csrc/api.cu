@@ -1,6 +1,7 @@
 // extern "C" boundary of the sr_gate library: argument validation and dispatch.
-// Every check runs on the host before anything is enqueued, so an error return
-// guarantees that no buffer was touched.
+// Every argument check runs on the host before anything is enqueued, so a validation
+// error guarantees that no buffer was touched; only SR_ERR_CUDA (a failed CUDA call or
+// launch) can arrive after earlier work of the same call is already on the stream.
 #include <stdio.h>
 #include <string.h>
 
@@ -16,7 +17,7 @@ void note_cuda_error(cudaError_t e, const char* where) {
              cudaGetErrorString(e));
 }
 
-static int check_gate_args(const int32_t* seqs, int32_t n_groups, int32_t N, int32_t stride,
+int check_gate_args(const int32_t* seqs, int32_t n_groups, int32_t N, int32_t stride,
                            int32_t K, int32_t norm_mode, const uint8_t* stop) {
     if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;
     if (stride < 0 || K < 0 || K > stride || K > SR_MAX_K) return SR_ERR_BAD_K;

@@ -71,7 +71,73 @@ __device__ __forceinline__ double pair_term(int d, int mi, int mj, int norm_mode
     return longer > 0 ? __ddiv_rn((double)d, (double)longer) : 0.0;
 }
 
+// d / L for 0 <= d, L <= 32 (0 when L == 0), correctly rounded: the compiler's constant
+// evaluation of an IEEE division equals the device's __ddiv_rn.  Terms of d_K for
+// prefixes of at most 32 symbols come from this table instead of a run-time division.
+struct QuotientTable {
+    double v[33 * 33];
+    constexpr QuotientTable() : v() {
+        for (int d = 0; d <= 32; ++d)
+            for (int l = 0; l <= 32; ++l) v[d * 33 + l] = l > 0 ? (double)d / (double)l : 0.0;
+    }
+};
+__device__ const QuotientTable kQuot = QuotientTable();
+
+// (i, j) of pair p, as i | j << 8, for every group size: filled in at compile time.
+struct PairTable {
+    uint16_t v[SR_MAX_N + 1][SR_MAX_N * (SR_MAX_N - 1) / 2];
+    constexpr PairTable() : v() {
+        for (int n = 2; n <= SR_MAX_N; ++n) {
+            int p = 0;
+            for (int i = 0; i < n; ++i)
+                for (int j = i + 1; j < n; ++j) v[n][p++] = (uint16_t)(i | (j << 8));
+        }
+    }
+};
+__device__ const PairTable kPairs = PairTable();
+
+// One column of the bit-vector edit-distance recurrence on a single 32-bit word of
+// vertical deltas (Pv: +1, Mv: -1), horizontal input +1 at row 0.  `Ph` / `Mh` return the
+// horizontal delta words BEFORE the shift (bit r = delta leaving row r).
+__device__ __forceinline__ void word_column(uint32_t Eq, uint32_t& Pv, uint32_t& Mv,
+                                            uint32_t& Ph, uint32_t& Mh) {
+    const uint32_t Xv = Eq | Mv;
+    const uint32_t Xh = (((Eq & Pv) + Pv) ^ Pv) | Eq;
+    Ph = Mv | ~(Xh | Pv);
+    Mh = Pv & Xh;
+    const uint32_t Phs = (Ph << 1) | 1u;
+    const uint32_t Mhs = Mh << 1;
+    Pv = Mhs | ~(Xv | Phs);
+    Mv = Phs & Xv;
+}
+
+// Ordered fp64 sum of the P terms of a group (pair order), the integer sum of the raw
+// distances, the division by P and the strict comparison of Eq. 2, by one thread.  The
+// loads run eight ahead of the (necessarily sequential) additions.
+__device__ __forceinline__ void group_sum_and_gate(const double* term, const int32_t* dist, int P,
+                                                   const GateArgs& a, size_t g) {
+    double s = 0.0;
+    int isum = 0, p = 0;
+    for (; p + 8 <= P; p += 8) {
+        double t[8];
+        int d[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { t[u] = term[p + u]; d[u] = dist[p + u]; }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { s = __dadd_rn(s, t[u]); isum += d[u]; }
+    }
+    for (; p < P; ++p) { s = __dadd_rn(s, term[p]); isum += dist[p]; }
+    const double dk = __ddiv_rn(s, (double)P);
+    if (a.pair_sum) a.pair_sum[g] = isum;
+    if (a.mean) a.mean[g] = dk;
+    a.stop[g] = dk < a.threshold ? 1 : 0;
+}
+
 size_t align_up(size_t x, size_t a);
+
+// api.cu: the argument rules shared by every gate entry point (SR_OK or an SR_ERR_* code).
+int check_gate_args(const int32_t* seqs, int32_t n_groups, int32_t N, int32_t stride, int32_t K,
+                    int32_t norm_mode, const uint8_t* stop);
 
 // Device arena of the host-buffer entry points (api.cu): staged inputs, outputs, gate workspace.
 struct HostArena {

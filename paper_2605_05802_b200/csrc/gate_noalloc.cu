@@ -5,8 +5,10 @@
 // start-up, the trainer's allocator owns the rest, and a cudaMalloc from a helper
 // library either fails or fragments somebody's pool (and synchronises the device
 // at the worst moment, in the middle of a generation step).  For those callers the
-// multi-word gate's scratch lives in the array below, which the CUDA runtime sets
-// aside when the library is loaded on a GPU and releases at process exit.
+// multi-word gate's scratch lives in the array below.  It is part of this file's device
+// image: the CUDA runtime sets it aside on a GPU when that image is first loaded there --
+// with the runtime's default lazy loading that is the first call below on that device --
+// and releases it at process exit.
 #include <mutex>
 
 #include "common.cuh"
@@ -15,7 +17,7 @@ namespace sr {
 namespace {
 
 // Scratch of the multi-word pipeline (control block, pair descriptors, match
-// streams, ordering).  Held by every GPU that loads the library, until exit.
+// streams, ordering).  Held, until exit, by every GPU on which the entry point has run.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[SR_NOALLOC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
@@ -23,18 +25,23 @@ std::mutex g_mu;
 void* g_scratch_addr[kMaxDevices] = {nullptr};
 
 // In host code `g_noalloc_scratch` names a host-side shadow, not device memory; the
-// device address has to be asked for, once per device, with that device current.
+// device address has to be asked for, once per device, with that device current.  The
+// answer is remembered per device index (devices beyond the table are simply asked every
+// time); a cudaDeviceReset invalidates it, so a process that resets a device must not
+// call this entry point on it afterwards.
 int scratch_address(void** out) {
     int dev = 0;
     SR_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= kMaxDevices) return SR_ERR_BAD_N;
+    const bool cached = dev >= 0 && dev < kMaxDevices;
     std::lock_guard<std::mutex> lock(g_mu);
-    if (g_scratch_addr[dev] == nullptr) {
-        void* p = nullptr;
-        SR_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
-        g_scratch_addr[dev] = p;
+    if (cached && g_scratch_addr[dev] != nullptr) {
+        *out = g_scratch_addr[dev];
+        return SR_OK;
     }
-    *out = g_scratch_addr[dev];
+    void* p = nullptr;
+    SR_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    if (cached) g_scratch_addr[dev] = p;
+    *out = p;
     return SR_OK;
 }
 
@@ -46,8 +53,9 @@ extern "C" int sr_gate_noalloc(const int32_t* seqs, const int32_t* lens, int32_t
                                int32_t* pair_dist, int32_t* pair_sum, double* mean, uint8_t* stop,
                                int32_t* status, void* stream) {
     using namespace sr;
-    if (n_groups < 0 || N < 2 || N > SR_MAX_N) return SR_ERR_BAD_N;
-    if (stride < 0 || K < 0 || K > stride || K > SR_MAX_K) return SR_ERR_BAD_K;
+    // every argument rule of sr_gate first, so that an invalid call reports its own error
+    const int bad = check_gate_args(seqs, n_groups, N, stride, K, norm_mode, stop);
+    if (bad != SR_OK) return bad;
     if (K <= 32 || n_groups == 0)      // the single-word path needs no scratch at all
         return sr_gate(seqs, lens, n_groups, N, stride, K, threshold, norm_mode, pair_dist, pair_sum,
                        mean, stop, status, nullptr, 0, stream);

@@ -103,17 +103,6 @@ struct IncrArgs {
     int off_dist, off_term;                                // shared-memory offsets
 };
 
-// d / L for 0 <= d, L <= 32 (0 when L == 0), correctly rounded: the compiler's
-// constant evaluation of an IEEE division equals the device's __ddiv_rn.
-struct QuotientTable {
-    double v[33 * 33];
-    constexpr QuotientTable() : v() {
-        for (int d = 0; d <= 32; ++d)
-            for (int l = 0; l <= 32; ++l) v[d * 33 + l] = l > 0 ? (double)d / (double)l : 0.0;
-    }
-};
-__device__ const QuotientTable kQuot = QuotientTable();
-
 // Bit r set iff action r of rollout `i` equals sym, for r < len.  `quads` points at the
 // group's stored actions ([8][N] int4); four actions per load; positions >= len are
 // masked off, so whatever those words hold does not matter.
@@ -131,19 +120,6 @@ __device__ __forceinline__ uint32_t match_mask(const int4* quads, int N, int i, 
     }
     return eq & low_mask(len);
 }
-
-// (i, j) of pair p for every group size: filled in at compile time.
-struct PairTable {
-    uint16_t v[SR_MAX_N + 1][SR_MAX_N * (SR_MAX_N - 1) / 2];
-    constexpr PairTable() : v() {
-        for (int n = 2; n <= SR_MAX_N; ++n) {
-            int p = 0;
-            for (int i = 0; i < n; ++i)
-                for (int j = i + 1; j < n; ++j) v[n][p++] = (uint16_t)(i | (j << 8));
-        }
-    }
-};
-__device__ const PairTable kPairs = PairTable();
 
 // One thread per pair, `gpb` groups per CTA.  Everything a pair needs (its state, the
 // two lengths, the two new actions, the header) is requested in one round of

@@ -39,9 +39,21 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_strerror_is_total(lib):
-    for code in range(-9, 1):
-        assert lib.sr_strerror(code)
-    assert b"unknown" in lib.sr_strerror(-99)
+    codes = {v for k, v in vars(binding).items() if k.startswith("SR_ERR_")} | {binding.SR_OK}
+    header = open(os.path.join(ROOT, "include", "sr_gate.h")).read()
+    declared = {int(m) for m in re.findall(r"#define SR_ERR_[A-Z_]+ \((-\d+)\)", header)} | {0}
+    assert codes == declared                      # the binding knows every code the header defines
+    fallback = lib.sr_strerror(-99)
+    assert b"unknown" in fallback
+    for code in codes:
+        text = lib.sr_strerror(code)
+        assert text and text != fallback, code
+
+
+def test_noalloc_limit_is_the_header_constant(lib):
+    header = open(os.path.join(ROOT, "include", "sr_gate.h")).read()
+    m = re.search(r"#define SR_NOALLOC_SCRATCH_BYTES \((\d+)u << (\d+)\)", header)
+    assert m and lib.sr_gate_noalloc_limit_bytes() == int(m.group(1)) << int(m.group(2))
 
 
 def test_gate_rejects_bad_arguments_before_any_launch(lib):

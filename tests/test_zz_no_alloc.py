@@ -7,9 +7,15 @@ reuses the same array with the previous call's leftovers in it.
 
 Collected last on purpose: a run that stops at the first failure has then already
 run every other test."""
+import os
+import subprocess
+import sys
+
 import numpy as np
 import pytest
 import torch
+
+import oracle
 
 import paper_2605_05802_b200 as sr
 from paper_2605_05802_b200 import binding, build, workloads as W
@@ -27,6 +33,10 @@ def test_noalloc_refuses_what_does_not_fit_before_touching_the_gpu():
     assert b"scratch" in lib.sr_strerror(rc)
     assert lib.sr_gate_noalloc(fake, None, 4, 1, 64, 64, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_BAD_N
     assert lib.sr_gate_noalloc(fake, None, 4, 8, 64, 65, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_BAD_K
+    # an invalid call reports its own error even when the problem would not fit either
+    assert lib.sr_gate_noalloc(fake, None, 1024, 8, 1024, 1024, 0.12, 7, None, None, None, fake, None, None) == binding.SR_ERR_BAD_MODE
+    assert lib.sr_gate_noalloc(None, None, 1024, 8, 1024, 1024, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_NULL
+    assert lib.sr_gate_noalloc(fake + 4, None, 1024, 8, 1024, 1024, 0.12, 0, None, None, None, fake, None, None) == binding.SR_ERR_ALIGN
 
 
 def _run(fn, w, thr, **extra):
@@ -59,8 +69,45 @@ def test_noalloc_matches_sr_gate_on_consecutive_calls():
         got = _run(sr.sr_gate_noalloc, w, 0.5)
         for a, b in zip(got, want):                 # integers and the fp64 d_K bit for bit
             assert a.dtype == b.dtype and np.array_equal(a.view(np.uint8), b.view(np.uint8))
+        for a, b in zip(got, oracle.gate(w.seqs, w.lens, w.K, 0.5, w.norm_mode)):   # and the definition itself
+            assert np.array_equal(a.view(np.uint8), b.view(np.uint8))
         assert 0 < want[3].sum() < G
     # the single-word path needs no scratch and is served as well
     w1 = W.agent_gate(K=15)
     for a, b in zip(_run(sr.sr_gate_noalloc, w1, 0.5), _run(sr.sr_gate, w1, 0.5)):
         assert np.array_equal(a.view(np.uint8), b.view(np.uint8))
+
+
+_FIRST_CALL = """
+import sys
+sys.path.insert(0, {root!r})
+import numpy as np, torch
+import oracle
+import paper_2605_05802_b200 as sr
+from paper_2605_05802_b200 import workloads as W
+w = W.token_gate(seed=21, n_groups=6, min_len=40, max_len=260, N=4)
+dev = torch.device("cuda:0")
+seqs, lens = torch.from_numpy(w.seqs).to(dev), torch.from_numpy(w.lens).to(dev)
+G, N, stride = w.seqs.shape
+pd = torch.empty((G, N * (N - 1) // 2), dtype=torch.int32, device=dev)
+stop = torch.empty(G, dtype=torch.uint8, device=dev)
+mean = torch.empty(G, dtype=torch.float64, device=dev)
+# the very first library call of this process is the entry point under test
+sr.sr_gate_noalloc(seqs, lens, w.K, 0.5, w.norm_mode, pair_dist=pd, mean=mean, stop=stop)
+torch.cuda.synchronize()
+opd, _, omean, ostop = oracle.gate(w.seqs, w.lens, w.K, 0.5, w.norm_mode)
+assert np.array_equal(pd.cpu().numpy(), opd)
+assert np.array_equal(mean.cpu().numpy().view(np.uint64), omean.view(np.uint64))
+assert np.array_equal(stop.cpu().numpy(), ostop)
+print("first-call ok")
+"""
+
+
+@pytest.mark.gpu
+def test_first_call_of_a_fresh_process_sets_the_scratch_up():
+    """The documented set-up happens inside the first call on a device: check it in a
+    process that has made no other library call before."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-c", _FIRST_CALL.format(root=root)], capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0 and "first-call ok" in out.stdout, out.stdout + out.stderr
