@@ -25,6 +25,23 @@
 //   finish   one thread per group: ordered fp64 sum of the normalised terms,
 //            threshold, outputs.
 //
+// Band (decide mode).  There prep also counts, per pair, the positions at which the two
+// prefixes differ (after the common prefix): that count plus the length difference is an
+// UPPER bound of the distance (substitute the differing positions, insert or delete the
+// rest), and the threshold caps how large a distance can still matter.  An optimal
+// alignment of distance <= ub never leaves the diagonals d = row - column with
+// |d| + |(m - n) - d| <= ub (Ukkonen's cut-off), so pairs whose bound is small run a
+// banded task, served by CTAs of their own within the dp launch: the pattern's 32-row blocks are grouped in stripes of R blocks, stripe g
+// lives on lane g mod T of a ring of T lanes and is advanced only over the columns where
+// the band crosses it; a stripe the band enters starts from +1 vertical deltas below the
+// stripe above it and a stripe whose upper neighbour the band has left takes +1
+// horizontal deltas from above -- both over-estimates of cells outside the band, which
+// leave every cell on an optimal path exact.  The distance is read from a running score
+// at the bottom of the last stripe.  A result within the bound is the exact distance; a
+// result above it only says "more than the bound".  (Banding the exact mode from the
+// mismatch count alone was built as well: 41 % fewer block-columns on the token-level
+// batch, but the banded tasks run at a lower rate and the net gain was a few percent.)
+//
 // Which rollout of a pair is the pattern is fixed by a round-robin tournament on the
 // indices, so that every pattern CTA of `prep` serves the same number of texts.
 #include "common.cuh"
@@ -42,6 +59,7 @@ constexpr uint32_t kLocMulti = 0x8000u;
 constexpr uint32_t kChainEnd = 0xFFFFu;
 constexpr int kDpWarpsPerCta = 4;
 constexpr uint32_t kBinMask = 0x3FFu;
+constexpr int32_t kCappedFlag = 0x40000000;   // decide mode: the pair's distance exceeds its cap
 constexpr int kStripShift = 12;
 constexpr uint32_t kNeedsDp = 0x80000000u;
 static_assert(kNumBins <= (int)kBinMask + 1, "bin index must fit its field");
@@ -51,7 +69,10 @@ struct PairDesc {          // 16 bytes
     uint32_t pat_row;      // g * N + pattern rollout
     uint32_t bin;          // bits 0..9 bin index; bits 12..21 stripped common prefix (symbols,
                            // a multiple of 4); bit 31 = pair needs the dp kernel
-    uint32_t lower;        // decide mode: a lower bound of the pair's distance
+    uint32_t lower;        // bits 0..15 a lower bound of the pair's distance (decide mode),
+                           // bits 16..31 an upper bound (mismatching positions + length
+                           // difference; in decide mode also capped by what the threshold
+                           // still allows): the band of the pair follows from it
 };
 
 struct Ctl {               // int32 control block in the workspace
@@ -61,6 +82,7 @@ struct Ctl {               // int32 control block in the workspace
     int32_t task_start[kNumBins + 1];          // first warp task of every bin
     int32_t task_counter;
     int32_t total_tasks;
+    int32_t task_counter_band;                 // the banded tasks' own launch
 };
 
 struct MultiWs {
@@ -105,17 +127,26 @@ __host__ __device__ inline void team_shape(int m, int min_tlog, int& tlog, int& 
 }
 
 // Class of a team shape.  T = 1, 2, 4, 8 with R = 1..6 fill slots log2(T) * 8 + R - 1; the
-// shapes of small batches, T = 16 with R = 1, 2 and T = 32 with R = 1, take slots 6, 7, 14.
+// shapes of small batches, T = 16 with R = 1, 2 and T = 32 with R = 1, take slots 6, 7, 14;
+// the banded shapes (ring of T = 4 or 8 lanes, stripes of R = 1..4 blocks) take slots 15, 22,
+// 23, 30, 31.
 __host__ __device__ inline int class_of(int tlog, int R) {
     if (tlog < 4) return tlog * 8 + (R - 1);
     return tlog == 4 ? 5 + R : 14;
+}
+__host__ __device__ inline bool is_band_class(int cls) {
+    return cls == 15 || cls == 22 || cls == 23 || cls == 30 || cls == 31;
 }
 __host__ __device__ inline void shape_of_class(int cls, int& tlog, int& R) {
     if ((cls & 7) < 6) { tlog = cls >> 3; R = (cls & 7) + 1; }
     else if (cls == 6) { tlog = 4; R = 1; }
     else if (cls == 7) { tlog = 4; R = 2; }
     else if (cls == 14) { tlog = 5; R = 1; }
-    else { tlog = 0; R = 1; }               // unused slots: no pair ever lands here
+    else if (cls == 15) { tlog = 2; R = 1; }
+    else if (cls == 22) { tlog = 3; R = 1; }
+    else if (cls == 23) { tlog = 3; R = 2; }
+    else if (cls == 30) { tlog = 3; R = 3; }
+    else { tlog = 3; R = 4; }               // 31
 }
 
 // Bins order the pairs by the estimated running time of their warp task (text
@@ -123,12 +154,51 @@ __host__ __device__ inline void shape_of_class(int cls, int& tlog, int& R) {
 // bucket, by team shape: all pairs of a bin share the shape and have text lengths
 // within a few percent, and warps that pull tasks in bin order start the longest
 // tasks first, which keeps the finishing times of the warps close together.
-__host__ __device__ inline int bin_of(int n, int tlog, int R) {
-    const int cost = (n + (4 << tlog)) * (14 * R + 20);
+__host__ __device__ inline int bin_of_cost(int cost, int cls) {
     const int max_cost = (SR_MAX_K + 32) * (14 * kMaxR + 20) + 1;
     int bucket = (int)(((long long)cost * kLenBuckets) / max_cost);
     bucket = bucket < 0 ? 0 : (bucket >= kLenBuckets ? kLenBuckets - 1 : bucket);
-    return (kLenBuckets - 1 - bucket) * kNumClasses + class_of(tlog, R);
+    return (kLenBuckets - 1 - bucket) * kNumClasses + cls;
+}
+
+// Diagonals d = row - column an optimal alignment of an m x n pair can visit when its
+// distance is at most ub: |d| + |(m - n) - d| <= ub.  At least two diagonals wide, so that
+// a stripe always starts while the stripe above it is still running.
+__host__ __device__ inline void band_of(int m, int n, int ub, int& dlo, int& dhi) {
+    const int D = m - n, aD = D < 0 ? -D : D;
+    int e = (ub - aD) >> 1;
+    if (e < 0) e = 0;
+    dlo = (D < 0 ? D : 0) - e;
+    dhi = (D > 0 ? D : 0) + e;
+    if (dhi == dlo) ++dhi;
+}
+
+// Shape and bin of a pair of m rows x n columns (what is left after the common prefix)
+// whose distance is at most ub.  The banded shapes serve bands of up to 32 R (T - 1)
+// diagonals; one is taken when its estimated lane-time is clearly below that of the full
+// shape (the estimates count instructions per quad of columns and lane).
+__host__ __device__ inline int shape_and_bin(int m, int n, int ub, int min_tlog) {
+    int tlog, R;
+    team_shape(m, min_tlog, tlog, R);
+    const int nq = (n + 3) >> 2;
+    const int full_time = (nq + (1 << tlog) - 1) * (14 * R + 14);
+    const int full_work = full_time << tlog;
+    int dlo, dhi;
+    band_of(m, n, ub, dlo, dhi);
+    const int w = dhi - dlo;
+    // banded tasks are few and run with the machine half empty, so their shapes favour a
+    // short task (many lanes, few blocks per lane) over the last bit of lane efficiency
+    int bcls = -1;
+    if (w <= 96) bcls = 15; else if (w <= 224) bcls = 22; else if (w <= 448) bcls = 23;
+    else if (w <= 672) bcls = 30; else if (w <= 896) bcls = 31;
+    if (bcls >= 0) {
+        int btl, bR;
+        shape_of_class(bcls, btl, bR);
+        const int G = (((m + 31) >> 5) + bR - 1) / bR;      // stripes
+        const int band_time = (nq + G - 1) * (14 * bR + 20);
+        if ((band_time << btl) * 8 < full_work * 7) return bin_of_cost(4 * band_time, bcls);
+    }
+    return bin_of_cost(4 * full_time, class_of(tlog, R));
 }
 
 __device__ __forceinline__ int clamp_len(const int32_t* lens, size_t idx, int K, bool& neg) {
@@ -175,8 +245,8 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
     unsigned long long* s_slot = reinterpret_cast<unsigned long long*>(smem);    // [hslots_max]
     uint32_t* s_next = reinterpret_cast<uint32_t*>(s_slot + hslots_max);         // [pitch]
     __shared__ int s_txt[SR_MAX_N], s_len[SR_MAX_N], s_qstart[SR_MAX_N + 1], s_absent[SR_MAX_N];
-    __shared__ int s_cp[SR_MAX_N];
-    // (At K = 1024 the 36 KB of dynamic plus these 528 bytes of static shared memory sit just
+    __shared__ int s_cp[SR_MAX_N], s_differ[SR_MAX_N];
+    // (At K = 1024 the 36 KB of dynamic plus these 656 bytes of static shared memory sit just
     // under the size at which six CTAs share an SM: 512 bytes more were measured to cost one
     // CTA per SM and a fifth of the kernel's speed.  Smaller tables with more CTAs per SM are
     // slower too: the probe length matters more than the residency.  Six CTAs of 256 threads
@@ -241,6 +311,7 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
                 s_txt[t] = j;
                 s_len[t] = n;
                 s_absent[t] = 0;
+                s_differ[t] = 0;
                 s_cp[t] = cp;
                 if (neg_t && a.status) atomicOr(a.status, SR_STATUS_NEG_LEN);
             }
@@ -304,6 +375,14 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
         const uint32_t l3 = pattern_lookup(sym.w, h3, v3, s_slot, s_next, hslots);
         reinterpret_cast<uint2*>(locs + idx * W.pitch)[q] = make_uint2(l0 | (l1 << 16), l2 | (l3 << 16));
         if (kBounds) {
+            // positions below both lengths whose symbol is not the pattern's symbol at the same
+            // place (a symbol with several occurrences may be counted although it matches: the
+            // count only has to be an upper bound of the mismatches)
+            const int both = min(m, s_len[t]) - 4 * q;       // columns of this quad below both lengths
+            const uint32_t c0 = 4u * (uint32_t)q;
+            const int differ = (both > 0 && l0 != c0) + (both > 1 && l1 != c0 + 1u) +
+                               (both > 2 && l2 != c0 + 2u) + (both > 3 && l3 != c0 + 3u);
+            if (differ) atomicAdd(&s_differ[t], differ);
             const int left = s_len[t] - 4 * q;           // columns of this quad that exist
             const int absent = (l0 == kLocNone) + (left > 1 && l1 == kLocNone) +
                                (left > 2 && l2 == kLocNone) + (left > 3 && l3 == kLocNone);
@@ -318,14 +397,16 @@ multi_prep_kernel(GateArgs a, unsigned char* ws, MultiWs W, int hslots_max, int3
         if (strip < 0) {                              // one prefix starts the other (or is empty)
             dist_out[idx] = abs(m - n);
             descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i), 0u,
-                                  (uint32_t)abs(m - n)};
+                                  (uint32_t)abs(m - n) | ((uint32_t)abs(m - n) << 16)};
         } else {
-            int tlog, R;
-            team_shape(m - strip, W.min_tlog, tlog, R);
-            const int bin = bin_of(n - strip, tlog, R);
+            // upper bound: substitute the differing positions, insert / delete the rest (only
+            // the decide mode bands its pairs: 0xFFFF stands for "no bound")
+            const int upper = kBounds ? s_differ[tid] + abs(m - n) : 0xFFFF;
+            const int bin = shape_and_bin(m - strip, n - strip, upper, W.min_tlog);
             const int lower = kBounds ? max(abs(m - n), s_absent[tid]) : 0;
             descs[idx] = PairDesc{(uint32_t)m | ((uint32_t)n << 16), (uint32_t)(g * N + i),
-                                  (uint32_t)bin | ((uint32_t)strip << kStripShift) | kNeedsDp, (uint32_t)lower};
+                                  (uint32_t)bin | ((uint32_t)strip << kStripShift) | kNeedsDp,
+                                  (uint32_t)lower | ((uint32_t)upper << 16)};
             if (kBounds) dist_out[idx] = lower;            // the bound kernel bins the pairs it keeps
             else atomicAdd(&ctl->hist[bin], 1);
         }
@@ -386,6 +467,7 @@ multi_order_kernel(const PairDesc* descs, int32_t* order, Ctl* ctl, int n_pairs)
             ctl->task_start[kNumBins] = task_start + own_tasks;
             ctl->total_tasks = task_start + own_tasks;
             ctl->task_counter = 0;
+            ctl->task_counter_band = 0;
         }
     }
     __syncthreads();
@@ -529,8 +611,152 @@ __device__ __noinline__ void dp_task(int tlog, int pos, bool valid, const PairDe
     if (valid && top) dist_out[idx] = n + part;
 }
 
+// A banded warp task: 32/T teams, one pair per team, the team's T lanes a ring.  The
+// pattern's blocks are grouped in stripes of R blocks; stripe g runs on lane g mod T over
+// the quads of text columns in which the band crosses it, one iteration behind stripe
+// g - 1, exactly like the lanes of the full task; when the band has left a stripe its lane
+// takes the stripe T places further down, which starts from +1 vertical deltas below the
+// stripe above; a stripe whose upper neighbour the band has left takes +1 horizontal
+// deltas from above.  A lane keeps the score at the bottom row of its stripe (started from
+// the stripe above plus the +1 deltas it is initialised with, then advanced by the
+// horizontal delta that leaves the stripe in every column); the pair's distance is that
+// score of the last stripe after the last column, less the vertical deltas of the rows
+// beyond the pattern's end.  A result above the pair's bound is reported as bound + 1 with
+// kCappedFlag.
+template <int R>
+__device__ __noinline__ void dp_task_band(int tlog, int pos, bool valid, const PairDesc* descs,
+                                             const int32_t* order, const uint16_t* locs,
+                                             const uint16_t* nexts, int pitch, int32_t* dist_out,
+                                             uint32_t two) {
+    const int lane = threadIdx.x & 31;
+    const int T = 1 << tlog;
+    const int lt = lane & (T - 1);
+    const int src = (lane & ~(T - 1)) | ((lt - 1) & (T - 1));      // the lane of the stripe above
+    int idx = 0, m_all = 0, m = 0, n = 0, strip = 0, ub = 0;
+    const uint2* loc4 = reinterpret_cast<const uint2*>(locs);
+    const uint16_t* nxt = nexts;
+    if (valid) {
+        idx = order[pos];
+        const PairDesc d = descs[idx];
+        strip = (int)((d.bin >> kStripShift) & 0x3FFu);
+        m_all = (int)(d.mn & 0xFFFFu);
+        m = m_all - strip;
+        n = (int)(d.mn >> 16) - strip;
+        ub = (int)(d.lower >> 16);
+        loc4 = reinterpret_cast<const uint2*>(locs + (size_t)idx * pitch + strip);
+        nxt = nexts + (size_t)d.pat_row * pitch;
+    }
+    int dlo, dhi;
+    band_of(m, n, ub, dlo, dhi);
+    const int nq = (n + 3) >> 2;                       // quads of text columns
+    const int G = valid ? (((m + 31) >> 5) + R - 1) / R : 0;       // stripes
+    int iters = valid ? nq + G - 1 : 0;
+    iters = __reduce_max_sync(0xFFFFFFFFu, iters);
+    // quads in which the band crosses stripe g: columns 32 R g - dhi .. 32 R (g + 1) - 1 - dlo
+    auto first_quad = [&](int g) { const int c = 32 * R * g - dhi; return c <= 0 ? 0 : c >> 2; };
+    auto last_quad = [&](int g) { return min((32 * R * (g + 1) - 1 - dlo) >> 2, nq - 1); };
+
+    int g = lt;                                        // the stripe this lane holds
+    int js = 0x7FFFFFFF, je = -1, above_end = -1;      // its iterations; last quad of the stripe above
+    if (g < G) {
+        js = first_quad(g) + g;
+        je = last_quad(g) + g;
+        above_end = g > 0 ? last_quad(g - 1) : -1;
+    }
+    uint32_t Pv[R], Mv[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) { Pv[r] = 0xFFFFFFFFu; Mv[r] = 0u; }
+    uint32_t outP[4] = {0u, 0u, 0u, 0u}, outM[4] = {0u, 0u, 0u, 0u};
+    uint32_t up = 0u, down = 0u;                       // +1 / -1 horizontal deltas seen at the stripe's bottom
+    int base = 0, before = 0;                          // score = base + up - down; score before the last quad
+    const uint2 none = make_uint2(kLocNone | (kLocNone << 16), kLocNone | (kLocNone << 16));
+    uint2 q_next = none;
+
+    for (int j = 0; j < iters; ++j) {
+        // delta words and score of the stripe above, as its lane left them one iteration ago
+        uint32_t inP[4], inM[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            inP[u] = __shfl_sync(0xFFFFFFFFu, outP[u], src);
+            inM[u] = __shfl_sync(0xFFFFFFFFu, outM[u], src);
+        }
+        const int above_before = __shfl_sync(0xFFFFFFFFu, before, src);
+        if (j > je && g < G) {                         // the band has left this stripe: take the next one
+            g += T;
+            if (g < G) {
+                js = first_quad(g) + g;
+                je = last_quad(g) + g;
+                above_end = last_quad(g - 1);
+#pragma unroll
+                for (int r = 0; r < R; ++r) { Pv[r] = 0xFFFFFFFFu; Mv[r] = 0u; }
+            } else {
+                js = 0x7FFFFFFF;
+                je = -1;
+            }
+        }
+        if (j >= js && j <= je) {
+            const int qi = j - g;
+            uint2 q = q_next;
+            if (j == js) {
+                // first quad of the stripe: the rows start one apart below the stripe above
+                // (or below the matrix's first column)
+                q = __ldg(loc4 + qi);
+                base = qi > 0 ? above_before + 32 * R : 32 * R * (g + 1);
+                up = 0u;
+                down = 0u;
+            }
+            if (g == 0 || qi > above_end) {            // nothing above: row 0, or the band left it
+#pragma unroll
+                for (int u = 0; u < 4; ++u) { inP[u] = 0x80000000u; inM[u] = 0u; }
+            }
+            before = base + (int)up - (int)down;
+            const uint32_t rowabs = (uint32_t)(strip + 32 * R * g);
+            const int left = n - 4 * qi;               // columns of this quad that exist (>= 1)
+            column_step<R>(q.x & 0xFFFFu, rowabs, m_all, nxt, Pv, Mv, inP[0], inM[0], two);
+            up = __umulhi(inP[0], two) + up;           // top bit of the word: the delta leaving the stripe
+            down = __umulhi(inM[0], two) + down;
+            if (left > 1) {
+                column_step<R>(q.x >> 16, rowabs, m_all, nxt, Pv, Mv, inP[1], inM[1], two);
+                up = __umulhi(inP[1], two) + up;
+                down = __umulhi(inM[1], two) + down;
+            }
+            if (left > 2) {
+                column_step<R>(q.y & 0xFFFFu, rowabs, m_all, nxt, Pv, Mv, inP[2], inM[2], two);
+                up = __umulhi(inP[2], two) + up;
+                down = __umulhi(inM[2], two) + down;
+            }
+            if (left > 3) {
+                column_step<R>(q.y >> 16, rowabs, m_all, nxt, Pv, Mv, inP[3], inM[3], two);
+                up = __umulhi(inP[3], two) + up;
+                down = __umulhi(inM[3], two) + down;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { outP[u] = inP[u]; outM[u] = inM[u]; }
+            if (g == G - 1 && qi == nq - 1) {
+                // the score at the stripe's bottom row, less the vertical deltas of the rows
+                // past the pattern's end
+                int d = base + (int)up - (int)down;
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const int rows = min(max(m - 32 * (R * g + r), 0), 32);
+                    const uint32_t past = ~low_mask(rows);
+                    d -= __popc(Pv[r] & past) - __popc(Mv[r] & past);
+                }
+                dist_out[idx] = d > ub ? ((ub + 1) | kCappedFlag) : d;
+            }
+        }
+        q_next = (j + 1 > js && j + 1 <= je) ? __ldg(loc4 + (j + 1 - g)) : none;
+    }
+}
+
+// Persistent warps pull warp tasks, longest first, from the bins' task list.  kBoth: the
+// batch has banded tasks as well (decide mode); CTAs with an odd index then serve those,
+// from a task counter of their own, and the even CTAs the full tasks, so that the two
+// kinds -- neither of which fills the machine -- run side by side.
+template <bool kBoth>
 __global__ void __launch_bounds__(kDpWarpsPerCta * 32)
 multi_dp_kernel(unsigned char* ws, MultiWs W, int32_t* dist_out, uint32_t two) {
+    const bool kBand = kBoth && (blockIdx.x & 1);
     Ctl* ctl = reinterpret_cast<Ctl*>(ws + W.off_ctl);
     const PairDesc* descs = reinterpret_cast<const PairDesc*>(ws + W.off_desc);
     const int32_t* order = reinterpret_cast<const int32_t*>(ws + W.off_order);
@@ -538,9 +764,10 @@ multi_dp_kernel(unsigned char* ws, MultiWs W, int32_t* dist_out, uint32_t two) {
     const uint16_t* nexts = reinterpret_cast<const uint16_t*>(ws + W.off_next);
     const int lane = threadIdx.x & 31;
     const int total = ctl->total_tasks;
+    int32_t* counter = kBand ? &ctl->task_counter_band : &ctl->task_counter;
     while (true) {
         int task = 0;
-        if (lane == 0) task = atomicAdd(&ctl->task_counter, 1);
+        if (lane == 0) task = atomicAdd(counter, 1);
         task = __shfl_sync(0xFFFFFFFFu, task, 0);
         if (task >= total) break;
         int k = 0, hi = kNumBins;                     // last bin whose first task is <= task
@@ -548,18 +775,28 @@ multi_dp_kernel(unsigned char* ws, MultiWs W, int32_t* dist_out, uint32_t two) {
             const int mid = (k + hi) >> 1;
             if (ctl->task_start[mid] <= task) k = mid; else hi = mid;
         }
+        if (is_band_class(k % kNumClasses) != kBand) continue;
         int tlog, R;
         shape_of_class(k % kNumClasses, tlog, R);
         const int tpw = 32 >> tlog;
         const int pos = ctl->start[k] + (task - ctl->task_start[k]) * tpw + (lane >> tlog);
         const bool valid = pos < ctl->start[k] + ctl->fill[k];     // fill = pairs in the bin
-        switch (R) {
-            case 1: dp_task<1>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
-            case 2: dp_task<2>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
-            case 3: dp_task<3>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
-            case 4: dp_task<4>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
-            case 5: dp_task<5>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
-            default: dp_task<6>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+        if (kBand) {
+            switch (R) {
+                case 1: dp_task_band<1>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+                case 2: dp_task_band<2>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+                case 3: dp_task_band<3>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+                default: dp_task_band<4>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+            }
+        } else {
+            switch (R) {
+                case 1: dp_task<1>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+                case 2: dp_task<2>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+                case 3: dp_task<3>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+                case 4: dp_task<4>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+                case 5: dp_task<5>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+                default: dp_task<6>(tlog, pos, valid, descs, order, locs, nexts, W.pitch, dist_out, two); break;
+            }
         }
     }
 }
@@ -570,8 +807,14 @@ multi_dp_kernel(unsigned char* ws, MultiWs W, int32_t* dist_out, uint32_t two) {
 // is monotone, so the result is <= the true d_K.  If it is already not below the
 // threshold, the gate's answer is "continue" whatever the exact distances are: the
 // group is finished here and its pairs never reach the bit-vector kernel.
+// A group the bounds leave open still has a budget: with every other pair at its lower
+// bound, pair p can only keep d_K below the threshold while its distance stays at or below
+//     cap_p = L_p * (P * d_L - sum of the other pairs' bounded terms)
+// (L_p the longer prefix, 1 for raw distances).  The pair's band is cut to that cap (plus a
+// margin of two that swamps the rounding of this estimate); a pair whose banded result
+// exceeds its cap is reported as "more than the cap", which is all Eq. 2 needs to know.
 __global__ void __launch_bounds__(128)
-multi_bound_kernel(GateArgs a, PairDesc* descs, Ctl* ctl, uint8_t* flag, uint8_t* exact) {
+multi_bound_kernel(GateArgs a, PairDesc* descs, Ctl* ctl, uint8_t* flag, uint8_t* exact, int min_tlog) {
     const int g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= a.n_groups) return;
     const int N = a.N, P = pairs_of(N);
@@ -580,7 +823,7 @@ multi_bound_kernel(GateArgs a, PairDesc* descs, Ctl* ctl, uint8_t* flag, uint8_t
     int isum = 0;
     for (int p = 0; p < P; ++p) {
         const int m = (int)(d[p].mn & 0xFFFFu), n = (int)(d[p].mn >> 16);
-        const int lb = (int)d[p].lower;
+        const int lb = (int)(d[p].lower & 0xFFFFu);
         isum += lb;
         s = __dadd_rn(s, pair_term(lb, m, n, a.norm_mode));      // max(m, n) is symmetric in the roles
     }
@@ -589,8 +832,23 @@ multi_bound_kernel(GateArgs a, PairDesc* descs, Ctl* ctl, uint8_t* flag, uint8_t
     flag[g] = open ? 1 : 0;
     if (exact) exact[g] = open ? 1 : 0;
     if (open) {
-        for (int p = 0; p < P; ++p)
-            if (d[p].bin & kNeedsDp) atomicAdd(&ctl->hist[d[p].bin & kBinMask], 1);
+        const double budget = (double)P * a.threshold;
+        for (int p = 0; p < P; ++p) {
+            if (!(d[p].bin & kNeedsDp)) continue;
+            const int m = (int)(d[p].mn & 0xFFFFu), n = (int)(d[p].mn >> 16);
+            const int lb = (int)(d[p].lower & 0xFFFFu);
+            int ub = (int)(d[p].lower >> 16);
+            const double longer = a.norm_mode == SR_NORM_NONE ? 1.0 : (double)max(m, n);
+            const double room = (budget - (s - pair_term(lb, m, n, a.norm_mode))) * longer;
+            // room < 2^31 here: an open group has s < budget, so room <= (budget + term) * longer
+            const int cap = max(lb, (int)fmin(room, 1.0e9)) + 2;
+            ub = min(ub, cap);
+            const int strip = (int)((d[p].bin >> kStripShift) & 0x3FFu);
+            const int bin = shape_and_bin(m - strip, n - strip, ub, min_tlog);
+            d[p].bin = (uint32_t)bin | ((uint32_t)strip << kStripShift) | kNeedsDp;
+            d[p].lower = (uint32_t)lb | ((uint32_t)ub << 16);
+            atomicAdd(&ctl->hist[bin], 1);
+        }
     } else {
         for (int p = 0; p < P; ++p) d[p].bin &= ~kNeedsDp;
         if (a.pair_sum) a.pair_sum[g] = isum;
@@ -605,7 +863,7 @@ multi_bound_kernel(GateArgs a, PairDesc* descs, Ctl* ctl, uint8_t* flag, uint8_t
 constexpr int kFinishThreads = 256;
 
 __global__ void __launch_bounds__(kFinishThreads)
-multi_finish_kernel(GateArgs a, const int32_t* dist, const uint8_t* flag, int gpb) {
+multi_finish_kernel(GateArgs a, int32_t* dist, const uint8_t* flag, uint8_t* exact, int gpb) {
     __shared__ double s_term[kFinishThreads];
     __shared__ int32_t s_dist[kFinishThreads];
     const int N = a.N, P = pairs_of(N);
@@ -620,8 +878,11 @@ multi_finish_kernel(GateArgs a, const int32_t* dist, const uint8_t* flag, int gp
             bool neg = false;
             const int mi = clamp_len(a.lens, (size_t)(g0 + g) * N + i, a.K, neg);
             const int mj = clamp_len(a.lens, (size_t)(g0 + g) * N + j, a.K, neg);
-            const int d = dist[(size_t)g0 * P + tid];
-            s_dist[tid] = d;
+            // decide mode marks a distance beyond its pair's cap: the value is then a lower bound
+            const int raw = dist[(size_t)g0 * P + tid];
+            const int d = raw & ~kCappedFlag;
+            if (raw != d) dist[(size_t)g0 * P + tid] = d;
+            s_dist[tid] = raw;
             s_term[tid] = pair_term(d, mi, mj, a.norm_mode);
         }
         __syncthreads();
@@ -629,15 +890,17 @@ multi_finish_kernel(GateArgs a, const int32_t* dist, const uint8_t* flag, int gp
             const int g = g0 + tid;
             if (flag && flag[g] == 0) return;                // decided from the bounds
             double s = 0.0;
-            int isum = 0;
+            int isum = 0, capped = 0;
             for (int p = 0; p < P; ++p) {
                 s = __dadd_rn(s, s_term[tid * P + p]);
-                isum += s_dist[tid * P + p];
+                isum += s_dist[tid * P + p] & ~kCappedFlag;
+                capped |= s_dist[tid * P + p] & kCappedFlag;
             }
             const double dk = __ddiv_rn(s, (double)P);
             if (a.pair_sum) a.pair_sum[g] = isum;
             if (a.mean) a.mean[g] = dk;
             a.stop[g] = dk < a.threshold ? 1 : 0;
+            if (capped && exact) exact[g] = 0;          // some distances are lower bounds
         }
         return;
     }
@@ -647,12 +910,15 @@ multi_finish_kernel(GateArgs a, const int32_t* dist, const uint8_t* flag, int gp
     if (flag && flag[g] == 0) return;
     bool neg = false;
     double s = 0.0;
-    int isum = 0, p = 0;
+    int isum = 0, p = 0, capped = 0;
     for (int i = 0; i < N; ++i) {
         const int mi = clamp_len(a.lens, (size_t)g * N + i, a.K, neg);
         for (int j = i + 1; j < N; ++j, ++p) {
             const int mj = clamp_len(a.lens, (size_t)g * N + j, a.K, neg);
-            const int d = dist[(size_t)g * P + p];
+            const int raw = dist[(size_t)g * P + p];
+            const int d = raw & ~kCappedFlag;
+            if (raw != d) dist[(size_t)g * P + p] = d;
+            capped |= raw & kCappedFlag;
             isum += d;
             s = __dadd_rn(s, pair_term(d, mi, mj, a.norm_mode));
         }
@@ -661,6 +927,7 @@ multi_finish_kernel(GateArgs a, const int32_t* dist, const uint8_t* flag, int gp
     if (a.pair_sum) a.pair_sum[g] = isum;
     if (a.mean) a.mean[g] = dk;
     a.stop[g] = dk < a.threshold ? 1 : 0;
+    if (capped && exact) exact[g] = 0;
 }
 
 }  // namespace
@@ -721,7 +988,7 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     }
     if (decide) {
         multi_bound_kernel<<<(a.n_groups + 127) / 128, 128, 0, s>>>(
-            a, reinterpret_cast<PairDesc*>(ws + W.off_desc), ctl, flag, exact);
+            a, reinterpret_cast<PairDesc*>(ws + W.off_desc), ctl, flag, exact, W.min_tlog);
         SR_LAUNCH_CHECK("multi_bound_kernel");
     }
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[1], s));
@@ -738,11 +1005,12 @@ int launch_gate_multi(const GateArgs& a, void* ws_, size_t ws_bytes, cudaStream_
     long long cap = (long long)sms * 3;
     int blocks = (int)(want < cap ? want : cap);
     if (blocks < 1) blocks = 1;
-    multi_dp_kernel<<<blocks, kDpWarpsPerCta * 32, 0, s>>>(ws, W, dist, 2u);
+    if (decide) multi_dp_kernel<true><<<2 * blocks, kDpWarpsPerCta * 32, 0, s>>>(ws, W, dist, 2u);
+    else multi_dp_kernel<false><<<blocks, kDpWarpsPerCta * 32, 0, s>>>(ws, W, dist, 2u);
     SR_LAUNCH_CHECK("multi_dp_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[3], s));
     const int fin_gpb = P <= kFinishThreads ? kFinishThreads / P : 1;
-    multi_finish_kernel<<<(a.n_groups + fin_gpb - 1) / fin_gpb, kFinishThreads, 0, s>>>(a, dist, flag, fin_gpb);
+    multi_finish_kernel<<<(a.n_groups + fin_gpb - 1) / fin_gpb, kFinishThreads, 0, s>>>(a, dist, flag, exact, fin_gpb);
     SR_LAUNCH_CHECK("multi_finish_kernel");
     if (ev) SR_CUDA_TRY(cudaEventRecord(ev[4], s));
     return SR_OK;

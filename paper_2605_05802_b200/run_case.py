@@ -6,7 +6,7 @@ device time.  Handy for profiling a single kernel:
         python -m paper_2605_05802_b200.run_case --case c3 --reps 3
 
 Cases: c1, c2, c2x128 (65536 groups x N=8, K=15), c3 (4096 groups x N=16), c3x16
-(65536 groups), c4 (token level), c4s (256 groups), c5 (streaming, --groups to
+(65536 groups), c4 (token level), c4s (256 groups), c4d (token level through sr_gate_decide at --threshold), c5 (streaming, --groups to
 shrink), adv (advantages, 4M groups), orr (OR rule, 4M groups), bstats (batch
 statistics, 4M groups), keep (kept-group index list, 4M groups), sig (Appendix-B
 signals, 65536 groups x N=16), packed (token level from packed host input, 256 groups).
@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--case", default="c3")
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--groups", type=int, default=0)
+    ap.add_argument("--threshold", type=float, default=0.3)
     args = ap.parse_args()
     dev = torch.device("cuda:0")
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -45,13 +46,14 @@ def main():
         torch.cuda.synchronize()
         times.append(a.elapsed_time(b) * 1e3)
 
-    if args.case in ("c1", "c2", "c2x128", "c3", "c3x16", "c4", "c4s"):
+    if args.case in ("c1", "c2", "c2x128", "c3", "c3x16", "c4", "c4s", "c4d"):
         w = {"c1": lambda: W.tiny_gate(), "c2": lambda: W.agent_gate(K=15),
              "c2x128": lambda: W.agent_gate(K=15, n_groups=args.groups or 65536),
              "c3": lambda: W.large_group_gate(n_groups=args.groups or 4096),
              "c3x16": lambda: W.large_group_gate(n_groups=65536),
              "c4": lambda: W.token_gate(n_groups=args.groups or 1024),
-             "c4s": lambda: W.token_gate(n_groups=256)}[args.case]()
+             "c4s": lambda: W.token_gate(n_groups=256),
+             "c4d": lambda: W.token_gate(n_groups=args.groups or 1024)}[args.case]()
         G, N, stride = w.seqs.shape
         seqs = torch.from_numpy(w.seqs).to(dev)
         lens = torch.from_numpy(w.lens).to(dev)
@@ -60,9 +62,15 @@ def main():
         stop = torch.empty(G, dtype=torch.uint8, device=dev)
         wsb = sr.sr_gate_workspace_bytes(G, N, stride, w.K)
         ws = torch.empty(wsb, dtype=torch.uint8, device=dev) if wsb else None
+        if args.case == "c4d":
+            ex = torch.empty(G, dtype=torch.uint8, device=dev)
+            call = lambda: sr.sr_gate_decide(seqs, lens, w.K, args.threshold, w.norm_mode, pair_sum=ps, mean=mean,
+                                             stop=stop, exact=ex, workspace=ws)
+        else:
+            call = lambda: sr.sr_gate(seqs, lens, w.K, w.threshold, w.norm_mode, pair_sum=ps, mean=mean,
+                                      stop=stop, workspace=ws)
         for _ in range(args.reps):
-            timed(lambda: sr.sr_gate(seqs, lens, w.K, w.threshold, w.norm_mode, pair_sum=ps, mean=mean,
-                                     stop=stop, workspace=ws))
+            timed(call)
         print(f"{w.name}: {G} groups x N={N}, K={w.K}: median {statistics.median(times):.1f} us, "
               f"{W.dp_cells(w.lens, w.K) / statistics.median(times) / 1e3:.0f} GCUPS, stopped {int(stop.sum())}")
     elif args.case == "c5":

@@ -268,13 +268,35 @@ def dp_cells(lens: np.ndarray, K: int) -> int:
     return int(((s1 * s1 - s2) // 2).sum())
 
 
-def word_columns(lens: np.ndarray, K: int, seqs: np.ndarray = None) -> int:
+def _band_units(rows: np.ndarray, cols: np.ndarray, ub: np.ndarray) -> np.ndarray:
+    """(column, 32-row block) units inside the band of a rows x cols matrix whose
+    distance is at most ub: diagonals d = row - column with |d| + |(rows - cols) - d| <= ub
+    (at least two diagonals).  Vectorised over pairs; loops over the columns."""
+    D = rows - cols
+    e = np.maximum((ub - np.abs(D)) // 2, 0)
+    dlo = np.minimum(D, 0) - e
+    dhi = np.maximum(D, 0) + e
+    dhi = np.where(dhi == dlo, dhi + 1, dhi)
+    total = np.zeros_like(rows)
+    for c in range(int(cols.max(initial=0))):
+        lo = np.maximum(c + dlo, 0)
+        hi = np.minimum(c + dhi, rows - 1)
+        ok = (c < cols) & (hi >= lo)
+        total += np.where(ok, hi // 32 - lo // 32 + 1, 0)
+    return total
+
+
+def word_columns(lens: np.ndarray, K: int, seqs: np.ndarray = None, band: bool = False) -> int:
     """Work units of the bit-vector method: the sum over unordered pairs of
     (text columns) x (32-row blocks of the pattern), taking for every pair the
     cheaper of the two orientations.  Used only to express roofline fractions.
     With ``seqs`` the common prefix of every pair, rounded down to a multiple of
     four symbols, is left out (nothing at all if one prefix contains the other):
-    the multi-word kernels never run those rows and columns."""
+    the multi-word kernels never run those rows and columns.  With ``band`` a pair
+    also counts no more than the units inside the band that its mismatch count
+    implies (differing positions after the common prefix + length difference is an
+    upper bound of the distance; an optimal alignment stays within the diagonals
+    that bound allows), again in the cheaper orientation."""
     m = np.minimum(np.maximum(lens.astype(np.int64), 0), K)
     total = 0
     N = lens.shape[1]
@@ -287,8 +309,19 @@ def word_columns(lens: np.ndarray, K: int, seqs: np.ndarray = None) -> int:
                 differs = (seqs[:, i, :] != seqs[:, j, :]) | (pos >= lo.reshape(-1, 1))
                 first = np.where(differs.any(axis=1), np.argmax(differs, axis=1), lo)
                 cut = np.where(first >= lo, np.maximum(a, b), first & ~3)
-                a, b = np.maximum(a - cut, 0), np.maximum(b - cut, 0)
-            total += int(np.minimum(a * ((b + 31) // 32), b * ((a + 31) // 32)).sum())
+                ra, rb = np.maximum(a - cut, 0), np.maximum(b - cut, 0)
+            else:
+                ra, rb = a, b
+            units = np.minimum(ra * ((rb + 31) // 32), rb * ((ra + 31) // 32))
+            if band and seqs is not None:
+                lo = np.minimum(a, b)
+                mism = ((seqs[:, i, :] != seqs[:, j, :]) & (pos < lo.reshape(-1, 1))).sum(axis=1)
+                ub = mism + np.abs(a - b)
+                live = (ra > 0) & (rb > 0)
+                banded = np.minimum(_band_units(np.where(live, ra, 0), np.where(live, rb, 0), ub),
+                                    _band_units(np.where(live, rb, 0), np.where(live, ra, 0), ub))
+                units = np.where(live, np.minimum(units, banded), units)
+            total += int(units.sum())
     return total
 
 

@@ -177,6 +177,74 @@ def test_multiword_shared_prefixes():
     assert want[0][1].max() == 1                           # second group: one substitution per pair
 
 
+def _edited_group(rng, base, N, subs, indels, vocab):
+    """N rollouts derived from `base`: `subs` substitutions each, then `indels` single-symbol
+    insertions or deletions at random places (lengths end up different)."""
+    rows = []
+    for _ in range(N):
+        r = list(base)
+        for p in rng.choice(len(r), size=min(subs, len(r)), replace=False):
+            r[p] = int(rng.integers(0, vocab))
+        for _ in range(indels):
+            p = int(rng.integers(0, len(r)))
+            if rng.random() < 0.5 and len(r) > 40:
+                del r[p]
+            else:
+                r.insert(p, int(rng.integers(0, vocab)))
+        rows.append(r)
+    return rows
+
+
+@pytest.mark.parametrize("vocab", [4, 50000])
+def test_multiword_banded_pairs(vocab):
+    """Pairs whose mismatch count bounds their distance well below their length run the
+    banded recurrence.  Bands of every shape (few to a few hundred diagonals), lengths
+    from two blocks to the maximum, equal and unequal lengths, edits bunched at the ends
+    or spread out, rollouts that differ in nothing but their last symbol, and a small
+    vocabulary whose repeats make the mismatch count loose and the occurrence chains long:
+    every distance is compared with the oracle."""
+    rng = np.random.default_rng(77 + vocab)
+    stride = 1024
+    groups = []
+    for L in (70, 130, 300, 640, 1000, 1024):
+        for subs, indels in ((1, 0), (3, 2), (L // 16, 0), (L // 8, 3), (L // 5, 8), (L // 3, 20)):
+            base = rng.integers(0, vocab, size=min(L, stride - 24)).tolist()
+            groups.append(_edited_group(rng, base, 5, subs, indels, vocab))
+    # edits bunched at the start / at the end of otherwise identical rollouts
+    base = rng.integers(0, vocab, size=900).tolist()
+    front = [[int(rng.integers(0, vocab)) for _ in range(k)] + base[k:] for k in (1, 5, 37, 64, 100)]
+    back = [base[:900 - k] + [int(rng.integers(0, vocab)) for _ in range(k)] for k in (1, 5, 37, 64, 100)]
+    grown = [base[:900 - k] for k in (0, 1, 31, 32, 200)]                   # prefixes of one another
+    shifted = [base[k:] + base[:k] for k in (0, 1, 2, 3, 40)]                # rotations: loose bound
+    groups += [front, back, grown, shifted]
+    G, N = len(groups), 5
+    seqs = np.zeros((G, N, stride), dtype=np.int32)
+    lens = np.zeros((G, N), dtype=np.int32)
+    for g, rows in enumerate(groups):
+        for i, r in enumerate(rows):
+            r = r[:stride]
+            seqs[g, i, :len(r)] = r
+            lens[g, i] = len(r)
+    want = oracle.gate(seqs, lens, stride, 0.1, threads=8)
+    got = gate_gpu(seqs, lens, stride, 0.1)
+    assert_gate_matches(got, want, f"banded pairs vocab={vocab}")
+    assert 0 < want[3].sum() < G
+
+
+def test_multiword_banded_full_size_converged_groups():
+    """The benchmark's recipe with every group converged (10 % substitutions): all long
+    equal-length pairs take the banded path, at the size the benchmark runs."""
+    w = W.token_gate(seed=5, n_groups=256)
+    seqs = w.seqs.copy()
+    conv = W.token_gate(seed=6, n_groups=256)
+    seqs[1::2] = conv.seqs[0::2][:128]                     # odd groups converged as well
+    lens = w.lens.copy()
+    lens[1::2] = conv.lens[0::2][:128]
+    want = oracle.gate(seqs, lens, w.K, 0.25, threads=16)
+    got = gate_gpu(seqs, lens, w.K, 0.25)
+    assert_gate_matches(got, want, "converged token groups")
+
+
 @pytest.mark.parametrize("N", [2, 3, 7, 8, 16, 32])
 def test_group_sizes(N):
     rng = np.random.default_rng(N)
@@ -306,15 +374,17 @@ def test_c5_incremental_ragged_termination():
     _check_stream(W.streaming_gate(n_groups=1024, ragged=True))
 
 
-def test_incremental_full_size_final_step():
+def test_incremental_full_size_every_step():
+    """The benchmark's own size (65 536 groups), compared with a recomputation from
+    scratch after every one of the 30 steps."""
     s = W.streaming_gate()
     inc = IncrementalGate(s.n_groups, s.N, max_steps=s.steps)
+    threads = min(16, oracle.max_threads())
     for t in range(s.steps):
         got = inc.step(s.actions[t], s.threshold, s.norm_mode)
-        if t in (0, 14, 29):
-            seqs, lens = W.stream_prefix(s.actions, t + 1)
-            want = oracle.gate(seqs, lens, 32, s.threshold, s.norm_mode, threads=8)
-            assert_gate_matches(got, want, f"C5 full step {t + 1}")
+        seqs, lens = W.stream_prefix(s.actions, t + 1)
+        want = oracle.gate(seqs, lens, 32, s.threshold, s.norm_mode, threads=threads)
+        assert_gate_matches(got, want, f"C5 full step {t + 1}")
 
 
 def test_incremental_other_group_sizes_overflow_and_snapshot():
