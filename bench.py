@@ -235,6 +235,26 @@ def main():
         sr.sr_gate(seqs, lens, K, w.threshold, w.norm_mode, pair_sum=ps, mean=mean, stop=stop, workspace=ws)
         sr.sr_grpo_advantage(rewards, stop, 1e-6, adv=adv, zero_var=zv)
 
+    # ---- before any timing: the outputs of this very configuration against the oracle on a
+    # sample of groups, at the paper's threshold and at one where the mask is mixed
+    verify = None
+    if rank == 0:
+        import oracle
+        cores = min(os.cpu_count() or 1, oracle.max_threads())
+        n_check = min(G, 96)
+        pd = torch.empty((G, P), dtype=torch.int32, device=dev)
+        verify = {"groups_checked": n_check, "thresholds": [], "cut_in_sample": []}
+    for thr in ((w.threshold, 0.5) if rank == 0 else ()):
+        sr.sr_gate(seqs, lens, K, thr, w.norm_mode, pair_dist=pd, pair_sum=ps, mean=mean, stop=stop, workspace=ws)
+        torch.cuda.synchronize()
+        o_pd, o_ps, o_mean, o_stop = oracle.gate(w.seqs[:n_check], w.lens[:n_check], K, thr, w.norm_mode, threads=cores)
+        assert np.array_equal(pd[:n_check].cpu().numpy(), o_pd), "pair distances differ from the oracle"
+        assert np.array_equal(ps[:n_check].cpu().numpy(), o_ps), "pair sums differ from the oracle"
+        assert np.array_equal(mean[:n_check].cpu().numpy().view(np.uint64), o_mean.view(np.uint64)), "d_K differs from the oracle"
+        assert np.array_equal(stop[:n_check].cpu().numpy(), o_stop), "stop mask differs from the oracle"
+        verify["thresholds"].append(thr)
+        verify["cut_in_sample"].append(int(o_stop.sum()))
+
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -337,6 +357,7 @@ def main():
                      "traffic": traffic_from_profiles("multi_dp_kernel", os.path.join(ROOT, "paper_2605_05802_b200", "csrc", "gate_multi.cu")),
                      "word_columns": wcols, "word_columns_before_prefix_removal": wcols_full,
                      "ms_per_launch": dp_ms},
+        "verified_against_oracle": verify,
     }
 
     # ------------------------------------------------ side measurements (1 GPU only)
@@ -352,6 +373,10 @@ def main():
         # issue on the FMA pipe, so the logic-only rate is the pipe's own ceiling
         line["roofline"]["peak_probe_logic"] = probe["logic"]
         line["roofline"]["frac_of_probe_logic"] = achieved / probe["logic"]
+        # the recurrence's own mix (8 logic : 2 add) measured register-only on this GPU: the
+        # adds also issue on the FMA pipe, so this ceiling is a little above the logic rate
+        line["roofline"]["peak_probe_mix"] = probe["mix8l2a"]
+        line["roofline"]["frac_of_probe_mix"] = achieved / probe["mix8l2a"]
 
         def gate_case(wl, reps=20):
             g, n, st = wl.seqs.shape
@@ -410,9 +435,15 @@ def main():
             per_group = Pn * 32 + s5.N * (4 * t_ + 4) + s5.N * 8 + s5.N * 4 + 9
             bytes_steps.append(per_group * s5.n_groups)
         gbs = [b / (ms * 1e-3) / 1e9 for b, ms in zip(bytes_steps, step_ms)]
+        # DP cells that are new at step t: every pair's matrix grows from (t-1)^2 to t^2 cells
+        new_cells = s5.n_groups * Pn * s5.steps * s5.steps
         extras["C5_stream"] = {"groups": s5.n_groups, "steps": s5.steps, "us_per_step_median": statistics.median(step_ms) * 1e3,
                                "us_total": sum(step_ms) * 1e3,
+                               "us_per_step": [round(x * 1e3, 1) for x in step_ms],
                                "group_gates_per_s": s5.n_groups * s5.steps / (sum(step_ms) * 1e-3),
+                               "new_cells_per_s": new_cells / (sum(step_ms) * 1e-3),
+                               "bytes_per_group_step": "28*32 pair state both ways + 8*(4t+4) stored actions read + append "
+                                                       "+ 8*8 lengths both ways + 8*4 new actions + 9 outputs",
                                "hbm_gbs_mean": statistics.mean(gbs), "hbm_gbs_last_step": gbs[-1],
                                "hbm_frac_mean": statistics.mean(gbs) / peaks["hbm_gbs"],
                                "hbm_peak_source": peaks["source"]}
@@ -437,6 +468,23 @@ def main():
                                "groups_per_s": G / (statistics.median(ms) * 1e-3),
                                "groups_computed_exactly": int(ex.sum().item()),
                                "note": "mask-equivalent mode; not the headline (work is skipped by design)"}
+        # the same mode at a threshold the bounds alone cannot settle: open groups run in bands
+        # cut to what the threshold still allows (compared with sr_gate's mask at that threshold)
+        thr_mid = 0.3
+        stop_ref = torch.empty(G, dtype=torch.uint8, device=dev)
+        ms_gate = timed(lambda: sr.sr_gate(seqs, lens, K, thr_mid, w.norm_mode, pair_sum=ps, mean=mean,
+                                           stop=stop_ref, workspace=ws), 10)
+        ms = timed(lambda: sr.sr_gate_decide(seqs, lens, K, thr_mid, w.norm_mode, pair_sum=ps, mean=mean,
+                                             stop=stop_d, exact=ex, workspace=ws), 10)
+        assert torch.equal(stop_d, stop_ref)
+        extras["decide_C4_thr0.3"] = {"groups": G, "us_median": statistics.median(ms) * 1e3,
+                                      "us_sr_gate_same_threshold": statistics.median(ms_gate) * 1e3,
+                                      "groups_computed_exactly": int(ex.sum().item()),
+                                      "groups_cut": int(stop_ref.sum().item()),
+                                      "note": "above about 0.35 most groups have to be computed anyway and sr_gate is the faster call"}
+        # restore the headline outputs for the checks below
+        sr.sr_gate(seqs, lens, K, w.threshold, w.norm_mode, pair_sum=ps, mean=mean, stop=stop, workspace=ws)
+        torch.cuda.synchronize()
         # end to end with the padded [groups][N][stride] host array instead of packed prefixes
         h_seqs = torch.from_numpy(w.seqs).pin_memory()
         h_lens = torch.from_numpy(w.lens).pin_memory()
@@ -487,8 +535,11 @@ def main():
         ms = timed(lambda: sr.sr_group_signals(s3, None, w3.K, unique_prefix_ratio=outs[0],
                                                unique_action_ratio=outs[1], action_entropy=outs[2],
                                                bigram_jaccard_mean=outs[3]), 5)
+        sig_bytes = w3.n_groups * (w3.N * 32 * 4 + 32)
         extras["group_signals_C3x16"] = {"groups": w3.n_groups, "N": w3.N, "us_median": statistics.median(ms) * 1e3,
-                                         "groups_per_s": w3.n_groups / (statistics.median(ms) * 1e-3)}
+                                         "groups_per_s": w3.n_groups / (statistics.median(ms) * 1e-3),
+                                         "hbm_gbs": sig_bytes / (statistics.median(ms) * 1e-3) / 1e9,
+                                         "bound": "instruction issue (hashing 480 bigrams per group); far from the HBM roofline"}
         l5 = torch.randint(0, 31, (big, 8), dtype=torch.int32, device=dev)
         m5 = torch.rand(big, dtype=torch.float64, device=dev)
         t5 = torch.empty(big, dtype=torch.float64, device=dev)
@@ -504,6 +555,21 @@ def main():
         bs_bytes = big * (8 * 4 + 1)
         extras["batch_stats_x64"] = {"groups": big, "us_median": med * 1e3, "hbm_gbs": bs_bytes / (med * 1e-3) / 1e9,
                                      "hbm_frac": bs_bytes / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        flags = (torch.rand(big, device=dev) < 0.2).to(torch.uint8)
+        kidx = torch.empty(big, dtype=torch.int32, device=dev)
+        kcnt = torch.empty(1, dtype=torch.int32, device=dev)
+        kws = torch.empty(sr.sr_kept_groups_workspace_bytes(big), dtype=torch.uint8, device=dev)
+        ms = timed(lambda: sr.sr_kept_groups(flags, z_, index=kidx, count=kcnt, workspace=kws), 10)
+        med = statistics.median(ms)
+        kept_bytes = big * 2 + int(kcnt.item()) * 4 + 4
+        extras["kept_groups_x64"] = {"groups": big, "kept": int(kcnt.item()), "us_median": med * 1e3,
+                                     "hbm_gbs": kept_bytes / (med * 1e-3) / 1e9,
+                                     "hbm_frac": kept_bytes / (med * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        # host link: the end-to-end step cannot beat the copy of its own input
+        ms = timed(lambda: arena[:h_sym.numel() * 4].view(torch.int32).copy_(h_sym, non_blocking=True), 10)
+        med = statistics.median(ms)
+        extras["h2d_link"] = {"bytes": h_sym.numel() * 4, "ms": med, "gbs": h_sym.numel() * 4 / (med * 1e-3) / 1e9,
+                              "note": "pinned host -> device copy of the packed symbols alone: the floor of the e2e step"}
         line["extras"] = extras
 
         # CPU baseline: the oracle as it stands on this machine's host cores
@@ -517,8 +583,27 @@ def main():
         oracle.advantage(w.rewards[:sample], o_stop_cpu, 1e-6)
         dt = time.perf_counter() - t0
         assert np.array_equal(o_stop_cpu, stop.cpu().numpy()[:sample])
+        one = max(8, sample // (2 * cores))
+        c_1 = W.dp_cells(w.lens[:one], K)
+        t0 = time.perf_counter()
+        oracle.gate(w.seqs[:one], w.lens[:one], K, w.threshold, w.norm_mode, threads=1)
+        dt1 = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": c_s / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"first {sample} of {G} groups, one pass, {dt:.1f} s"}
+                                "sample": f"first {sample} of {G} groups, one pass, {dt:.1f} s",
+                                "single_thread": {"value": c_1 / dt1 / 1e9, "unit": UNIT, "cores": 1,
+                                                  "sample": f"first {one} groups, one pass, {dt1:.1f} s"}}
+        # groups whose ordered fp64 d_K and exact rational d_K fall on different sides of the
+        # threshold (none expected: the two differ by about 1e-16)
+        razor = {}
+        for name, wl in (("C1", W.tiny_gate()), ("C1_normalised", W.tiny_gate(raw_threshold=False)),
+                         ("C2_K15", W.agent_gate(K=15)), ("C2_K30", W.agent_gate(K=30)),
+                         ("C3", W.large_group_gate()), ("C4", w)):
+            o_pd, _, _, o_st = oracle.gate(wl.seqs, wl.lens, wl.K, wl.threshold, wl.norm_mode, threads=cores)
+            razor[name] = int((oracle.exact_mask(o_pd, wl.lens, wl.K, wl.threshold, wl.norm_mode) != o_st).sum())
+        sq, ln = W.stream_prefix(s5.actions[:, :8192], s5.steps)
+        o_pd, _, _, o_st = oracle.gate(sq, ln, 32, s5.threshold, s5.norm_mode, threads=cores)
+        razor["C5_final_step_8192_groups"] = int((oracle.exact_mask(o_pd, ln, 32, s5.threshold, s5.norm_mode) != o_st).sum())
+        line["extras"]["razor_edge_groups"] = razor
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

@@ -160,35 +160,49 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
 }
 
 // Batch reductions (Section 4.5 dilution, Section 3.4 norm kept): grid-stride over the
-// trajectories, fp64 partial sums per thread, warp shuffles, one atomic per warp.
+// groups, fp64 partial sums per thread, warp shuffles, one set of atomics per CTA.
+// N = 8 (the paper's G): four groups per trip, a grid stride apart (so that consecutive
+// lanes read consecutive 32-byte rows), their eight 16-byte loads and four decision bytes
+// issued before any arithmetic; the last trip takes whatever is left of the four with
+// predicated loads.  Measured at 0.59 of the copy bandwidth: the warps wait on loads (17
+// stall cycles per issue) while the fp32 -> fp64 conversions of the exact squares keep the
+// conversion unit a third busy.  Tried and not faster: four consecutive groups per thread
+// (uncoalesced 16-byte loads), eight groups per trip, larger CTAs, more CTAs (the five
+// atomics per CTA start to cost from about 5000 CTAs on).
 __global__ void __launch_bounds__(256)
 batch_stats_kernel(const float* __restrict__ adv, const uint8_t* __restrict__ stop, int N,
                    int n_groups, bool vec4, unsigned long long* counts, double* sumsq) {
     double ss_all = 0.0, ss_kept = 0.0;
     unsigned z_all = 0, z_kept = 0, kept_groups = 0;
     const int stride = gridDim.x * blockDim.x;
-    int g = blockIdx.x * blockDim.x + threadIdx.x;
+    long long g = blockIdx.x * blockDim.x + threadIdx.x;     // 64-bit: g + 4 * stride may pass 2^31
     if (vec4 && N == 8) {
-        // the paper's group size: four groups per trip, their eight 16-byte loads issued
-        // before any arithmetic, zero tests in fp32 (exact), squares in fp64
-        for (; g + 3 * stride < n_groups; g += 4 * stride) {
+        for (; g < n_groups; g += 4LL * stride) {
             float4 v[4][2];
             unsigned char st[4];
+            bool have[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const float4* row = reinterpret_cast<const float4*>(adv + (size_t)(g + u * stride) * 8);
-                v[u][0] = __ldg(row);
-                v[u][1] = __ldg(row + 1);
-                st[u] = stop ? stop[g + u * stride] : 0;
+                const long long gg = g + (long long)u * stride;
+                have[u] = gg < n_groups;
+                v[u][0] = v[u][1] = make_float4(1.f, 1.f, 1.f, 1.f);
+                st[u] = 0;
+                if (have[u]) {
+                    const float4* row = reinterpret_cast<const float4*>(adv + (size_t)gg * 8);
+                    v[u][0] = __ldg(row);
+                    v[u][1] = __ldg(row + 1);
+                    st[u] = stop ? stop[gg] : 0;
+                }
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
+                if (!have[u]) continue;
                 const float f[8] = {v[u][0].x, v[u][0].y, v[u][0].z, v[u][0].w,
                                     v[u][1].x, v[u][1].y, v[u][1].z, v[u][1].w};
                 double ss = 0.0;
                 unsigned z = 0;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < 8; ++i) {        // zero tests in fp32 (exact), squares in fp64
                     const double a = (double)f[i];
                     ss += __dmul_rn(a, a);
                     z += f[i] == 0.0f;
@@ -201,7 +215,7 @@ batch_stats_kernel(const float* __restrict__ adv, const uint8_t* __restrict__ st
             }
         }
     }
-    for (; g < n_groups; g += stride) {            // one group per thread and trip
+    for (; g < n_groups; g += stride) {            // any other group size: one group per trip
         const bool kept = !(stop && stop[g]);
         kept_groups += kept;
         const float* row = adv + (size_t)g * N;
@@ -283,10 +297,10 @@ int launch_batch_stats(const float* adv, const uint8_t* stop, int32_t n_groups, 
     int dev = 0, sms = 0;
     SR_CUDA_TRY(cudaGetDevice(&dev));
     SR_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const bool vec4 = (N % 4 == 0) && (reinterpret_cast<uintptr_t>(adv) & 15) == 0;
     const int want = (n_groups + 255) / 256;
     const int cap = sms * 16;
     const int blocks = want < cap ? want : cap;
-    const bool vec4 = (N % 4 == 0) && (reinterpret_cast<uintptr_t>(adv) & 15) == 0;
     batch_stats_kernel<<<blocks, 256, 0, s>>>(adv, stop, N, n_groups, vec4,
                                               reinterpret_cast<unsigned long long*>(counts), sumsq);
     SR_LAUNCH_CHECK("batch_stats_kernel");
