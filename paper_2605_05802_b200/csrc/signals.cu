@@ -1,4 +1,6 @@
 // Further per-group signals of the paper's Appendix B and the OR-rule extension.
+#include <math.h>
+
 #include "common.cuh"
 
 namespace sr {
@@ -42,8 +44,8 @@ constexpr int kBgWords = 31;                    // 32 * 31 = 992 distinct bigram
 
 __global__ void __launch_bounds__(512)
 group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict__ lens, int N,
-                     int stride, int K, int slots, int slot_shift, double* upr, double* uar, double* ent,
-                     double* jac) {
+                     int stride, int K, int slots, int slot_shift, double ln_n, double* upr, double* uar,
+                     double* ent, double* jac) {
     __shared__ int32_t s_sym[SR_MAX_N * 33];
     __shared__ int32_t s_len[SR_MAX_N], s_raw[SR_MAX_N];
     __shared__ int32_t s_fp[SR_MAX_N], s_fa[SR_MAX_N], s_same[SR_MAX_N], s_card[SR_MAX_N];
@@ -150,7 +152,7 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
         }
         if (upr) upr[g] = __ddiv_rn((double)dp, (double)N);
         if (uar) uar[g] = __ddiv_rn((double)da, (double)N);
-        if (ent) ent[g] = __ddiv_rn(h, log((double)N));
+        if (ent) ent[g] = __ddiv_rn(h, ln_n);        // ln N comes from the host: one fp64 logarithm less in this serial tail
         if (jac) {
             double s = 0.0;
             for (int p = 0; p < P; ++p) s = __dadd_rn(s, s_term[p]);
@@ -283,8 +285,8 @@ int launch_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_gro
     while (slots < 2 * N * (K > 1 ? K - 1 : 1)) slots <<= 1;
     int slot_shift = 32;
     while ((1 << (32 - slot_shift)) < slots) --slot_shift;
-    group_signals_kernel<<<n_groups, threads, 0, s>>>(seqs, lens, N, stride, K, slots, slot_shift, upr,
-                                                      uar, ent, jac);
+    group_signals_kernel<<<n_groups, threads, 0, s>>>(seqs, lens, N, stride, K, slots, slot_shift,
+                                                      log((double)N), upr, uar, ent, jac);
     SR_LAUNCH_CHECK("group_signals_kernel");
     return SR_OK;
 }
