@@ -42,20 +42,33 @@ or_rule_kernel(const double* __restrict__ mean, const int32_t* __restrict__ lens
 constexpr int kBgSlots = 2048;                  // >= 2 * 32 rollouts * 31 bigrams
 constexpr int kBgWords = 31;                    // 32 * 31 = 992 distinct bigrams at most
 
+// Shared memory of a group, sized for the call's N and K (the arrays for 32 rollouts would
+// keep an SM at 8 CTAs whatever the group size): byte offsets into dynamic shared memory.
+struct SignalLayout {
+    int off_term, off_plogp, off_sym, off_owner, off_bits, off_small, off_bid, off_slot;
+    int words;                                  // words of a rollout's bigram bit set
+    int total;
+};
+
 __global__ void __launch_bounds__(512)
 group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict__ lens, int N,
-                     int stride, int K, int slots, int slot_shift, double ln_n, double* upr, double* uar,
-                     double* ent, double* jac) {
-    __shared__ int32_t s_sym[SR_MAX_N * 33];
-    __shared__ int32_t s_len[SR_MAX_N], s_raw[SR_MAX_N];
-    __shared__ int32_t s_fp[SR_MAX_N], s_fa[SR_MAX_N], s_same[SR_MAX_N], s_card[SR_MAX_N];
-    __shared__ uint32_t s_owner[kBgSlots];      // element (i * 32 + t) + 1 that claimed the slot
-    __shared__ uint16_t s_bid[kBgSlots];        // dense bigram id of a claimed slot
-    __shared__ uint16_t s_slot[SR_MAX_N * 32];  // slot of every element's bigram
-    __shared__ uint32_t s_bits[SR_MAX_N * kBgWords];
-    __shared__ int s_nbig;
-    __shared__ double s_term[SR_MAX_N * (SR_MAX_N - 1) / 2];
-    __shared__ double s_plogp[SR_MAX_N];
+                     int stride, int K, int slots, int slot_shift, double ln_n, SignalLayout L,
+                     double* upr, double* uar, double* ent, double* jac) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    double* s_term = reinterpret_cast<double*>(smem + L.off_term);          // [P]
+    double* s_plogp = reinterpret_cast<double*>(smem + L.off_plogp);        // [N]
+    int32_t* s_sym = reinterpret_cast<int32_t*>(smem + L.off_sym);          // [N][33]
+    uint32_t* s_owner = reinterpret_cast<uint32_t*>(smem + L.off_owner);    // [slots] element (i * 32 + t) + 1 that claimed the slot
+    uint32_t* s_bits = reinterpret_cast<uint32_t*>(smem + L.off_bits);      // [N][kBgWords]
+    int32_t* s_len = reinterpret_cast<int32_t*>(smem + L.off_small);        // 6 arrays of [N] and a counter
+    int32_t* s_raw = s_len + N;
+    int32_t* s_fp = s_raw + N;
+    int32_t* s_fa = s_fp + N;
+    int32_t* s_same = s_fa + N;
+    int32_t* s_card = s_same + N;
+    int& s_nbig = *(s_card + N);
+    uint16_t* s_bid = reinterpret_cast<uint16_t*>(smem + L.off_bid);        // [slots] dense bigram id of a claimed slot
+    uint16_t* s_slot = reinterpret_cast<uint16_t*>(smem + L.off_slot);      // [N * 32] slot of every element's bigram
     const int g = blockIdx.x, tid = threadIdx.x, nthr = blockDim.x;
     const int P = pairs_of(N);
     for (int i = tid; i < N; i += nthr) {
@@ -99,8 +112,8 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
     // one thread per unordered pair: equal prefixes / equal step-K actions knock out the
     // later rollout as a "first occurrence" and count towards the action's multiplicity
     for (int p = tid; p < P; p += nthr) {
-        int i, j;
-        pair_from_index(p, N, i, j);
+        const int pr = kPairs.v[N][p];
+        const int i = pr & 0xFF, j = pr >> 8;
         const int32_t* a = s_sym + i * 33;
         const int32_t* b = s_sym + j * 33;
         const int mi = s_len[i];
@@ -128,8 +141,8 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
         }
         __syncthreads();
         for (int p = tid; p < P; p += nthr) {
-            int i, j;
-            pair_from_index(p, N, i, j);
+            const int pr = kPairs.v[N][p];
+            const int i = pr & 0xFF, j = pr >> 8;
             int both = 0;
             for (int w = 0; w < words; ++w) both += __popc(s_bits[i * kBgWords + w] & s_bits[j * kBgWords + w]);
             const int uni = s_card[i] + s_card[j] - both;
@@ -285,8 +298,21 @@ int launch_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_gro
     while (slots < 2 * N * (K > 1 ? K - 1 : 1)) slots <<= 1;
     int slot_shift = 32;
     while ((1 << (32 - slot_shift)) < slots) --slot_shift;
-    group_signals_kernel<<<n_groups, threads, 0, s>>>(seqs, lens, N, stride, K, slots, slot_shift,
-                                                      log((double)N), upr, uar, ent, jac);
+    SignalLayout L;
+    int off = 0;
+    auto take = [&](int bytes) { int o = off; off = (off + bytes + 15) & ~15; return o; };
+    L.off_term = take(pairs_of(N) * 8);
+    L.off_plogp = take(N * 8);
+    L.off_sym = take(N * 33 * 4);
+    L.off_owner = take(slots * 4);
+    L.off_bits = take(N * kBgWords * 4);
+    L.off_small = take((6 * N + 1) * 4);
+    L.off_bid = take(slots * 2);
+    L.off_slot = take(N * 32 * 2);
+    L.words = kBgWords;
+    L.total = off;
+    group_signals_kernel<<<n_groups, threads, L.total, s>>>(seqs, lens, N, stride, K, slots, slot_shift,
+                                                            log((double)N), L, upr, uar, ent, jac);
     SR_LAUNCH_CHECK("group_signals_kernel");
     return SR_OK;
 }
