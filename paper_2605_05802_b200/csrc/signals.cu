@@ -41,6 +41,7 @@ or_rule_kernel(const double* __restrict__ mean, const int32_t* __restrict__ lens
 // the prefix / step-K-action comparisons; thread 0 adds everything up in a fixed order.
 constexpr int kBgSlots = 2048;                  // >= 2 * 32 rollouts * 31 bigrams
 constexpr int kBgWords = 31;                    // 32 * 31 = 992 distinct bigrams at most
+constexpr int kSymPitch = 36;                   // words per staged prefix: 32 + pad, rows 16-byte aligned
 
 // Shared memory of a group, sized for the call's N and K (the arrays for 32 rollouts would
 // keep an SM at 8 CTAs whatever the group size): byte offsets into dynamic shared memory.
@@ -57,7 +58,7 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
     extern __shared__ __align__(16) unsigned char smem[];
     double* s_term = reinterpret_cast<double*>(smem + L.off_term);          // [P]
     double* s_plogp = reinterpret_cast<double*>(smem + L.off_plogp);        // [N]
-    int32_t* s_sym = reinterpret_cast<int32_t*>(smem + L.off_sym);          // [N][33]
+    int32_t* s_sym = reinterpret_cast<int32_t*>(smem + L.off_sym);          // [N][kSymPitch]
     uint32_t* s_owner = reinterpret_cast<uint32_t*>(smem + L.off_owner);    // [slots] element (i * 32 + t) + 1 that claimed the slot
     uint32_t* s_bits = reinterpret_cast<uint32_t*>(smem + L.off_bits);      // [N][kBgWords]
     int32_t* s_len = reinterpret_cast<int32_t*>(smem + L.off_small);        // 6 arrays of [N] and a counter
@@ -83,27 +84,28 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
         const int i = e >> 3, q = e & 7;
         if (q < q4) {
             const int4 v = __ldg(reinterpret_cast<const int4*>(seqs + ((size_t)g * N + i) * stride) + q);
-            int32_t* d = s_sym + i * 33 + 4 * q;
-            d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+            *reinterpret_cast<int4*>(s_sym + i * kSymPitch + 4 * q) = v;
         }
     }
-    if (jac) {
-        for (int e = tid; e < slots; e += nthr) s_owner[e] = 0u;
-        for (int e = tid; e < N * kBgWords; e += nthr) s_bits[e] = 0u;
+    if (jac) {                                   // 16-byte stores: both regions are padded to 16 bytes
+        uint4* o4 = reinterpret_cast<uint4*>(s_owner);
+        for (int e = tid; e < slots / 4; e += nthr) o4[e] = make_uint4(0u, 0u, 0u, 0u);
+        uint4* b4 = reinterpret_cast<uint4*>(s_bits);
+        for (int e = tid; e < (N * kBgWords + 3) / 4; e += nthr) b4[e] = make_uint4(0u, 0u, 0u, 0u);
     }
     __syncthreads();
     if (jac) {                                   // bigram (a[t], a[t+1]) of rollout i -> slot
         for (int e = tid; e < N * 32; e += nthr) {
             const int i = e >> 5, t = e & 31;
             if (t + 1 >= s_len[i]) continue;
-            const int32_t x = s_sym[i * 33 + t], y = s_sym[i * 33 + t + 1];
+            const int32_t x = s_sym[i * kSymPitch + t], y = s_sym[i * kSymPitch + t + 1];
             uint32_t h = (((uint32_t)x * 0x9E3779B1u) ^ ((uint32_t)y * 0x85EBCA77u)) >> slot_shift;
             for (int probe = 0; probe < slots; ++probe) {         // at most half of the slots fill up
                 uint32_t o = s_owner[h];
                 if (o == 0u) o = atomicCAS(&s_owner[h], 0u, (uint32_t)e + 1u);
                 if (o == 0u) { s_bid[h] = (uint16_t)atomicAdd(&s_nbig, 1); break; }
                 const int oi = (int)(o - 1u) >> 5, ot = (int)(o - 1u) & 31;
-                if (s_sym[oi * 33 + ot] == x && s_sym[oi * 33 + ot + 1] == y) break;
+                if (s_sym[oi * kSymPitch + ot] == x && s_sym[oi * kSymPitch + ot + 1] == y) break;
                 h = (h + 1u) & (uint32_t)(slots - 1);
             }
             s_slot[e] = (uint16_t)h;
@@ -114,11 +116,15 @@ group_signals_kernel(const int32_t* __restrict__ seqs, const int32_t* __restrict
     for (int p = tid; p < P; p += nthr) {
         const int pr = kPairs.v[N][p];
         const int i = pr & 0xFF, j = pr >> 8;
-        const int32_t* a = s_sym + i * 33;
-        const int32_t* b = s_sym + j * 33;
+        const int32_t* a = s_sym + i * kSymPitch;
+        const int32_t* b = s_sym + j * kSymPitch;
         const int mi = s_len[i];
         bool same_p = mi == s_len[j];
-        for (int r = 0; same_p && r < mi; ++r) same_p = a[r] == b[r];
+        for (int q = 0; same_p && 4 * q < mi; ++q) {          // four symbols per 16-byte load
+            const int4 u = reinterpret_cast<const int4*>(a)[q], v = reinterpret_cast<const int4*>(b)[q];
+            const int left = mi - 4 * q;                     // symbols of this quad inside the prefix
+            same_p = u.x == v.x && (left < 2 || u.y == v.y) && (left < 3 || u.z == v.z) && (left < 4 || u.w == v.w);
+        }
         const bool has_i = s_raw[i] >= K && K >= 1, has_j = s_raw[j] >= K && K >= 1;
         const bool same_a = has_i == has_j && (!has_i || a[K - 1] == b[K - 1]);
         if (same_p) s_fp[j] = 0;
@@ -303,7 +309,7 @@ int launch_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_gro
     auto take = [&](int bytes) { int o = off; off = (off + bytes + 15) & ~15; return o; };
     L.off_term = take(pairs_of(N) * 8);
     L.off_plogp = take(N * 8);
-    L.off_sym = take(N * 33 * 4);
+    L.off_sym = take(N * kSymPitch * 4);
     L.off_owner = take(slots * 4);
     L.off_bits = take(N * kBgWords * 4);
     L.off_small = take((6 * N + 1) * 4);
