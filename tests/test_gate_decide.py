@@ -120,3 +120,27 @@ def test_decide_computes_open_groups_in_capped_bands(thr):
     assert (ps[lo] == pd[lo].sum(axis=1)).all()
     assert (mean[lo] <= omean[lo]).all() and (mean[lo] >= thr).all()
     assert stop[ex].sum() == ostop.sum()                  # every cut group was computed exactly
+
+
+@pytest.mark.gpu
+def test_decide_large_groups_and_raw_distances():
+    """Groups of 32 rollouts (496 pairs: the finish pass takes its one-thread-per-group path)
+    and the raw-distance normalisation, at thresholds that leave groups open."""
+    big = W.token_gate(seed=21, n_groups=6, min_len=40, max_len=130, N=32)
+    for thr in (0.15, 0.4, 0.8):
+        opd, ops, omean, ostop = oracle.gate(big.seqs, big.lens, big.K, thr, big.norm_mode, threads=8)
+        pd, ps, mean, stop, exact = _run_decide(big, thr, big.norm_mode)
+        assert np.array_equal(stop, ostop)
+        ex = exact == 1
+        assert np.array_equal(pd[ex], opd[ex]) and np.array_equal(mean[ex].view(np.uint64), omean[ex].view(np.uint64))
+        assert (pd[~ex] <= opd[~ex]).all() and (stop[~ex] == 0).all()
+    w = W.token_gate(seed=22, n_groups=40, min_len=60, max_len=400)
+    for thr in (30.0, 120.0, 300.0):                                    # thresholds on the raw mean distance
+        opd, ops, omean, ostop = oracle.gate(w.seqs, w.lens, w.K, thr, 1, threads=8)
+        pd, ps, mean, stop, exact = _run_decide(w, thr, 1)
+        assert np.array_equal(stop, ostop)
+        ex = exact == 1
+        assert np.array_equal(pd[ex], opd[ex]) and np.array_equal(ps[ex], ops[ex])
+        assert np.array_equal(mean[ex].view(np.uint64), omean[ex].view(np.uint64))
+        assert (pd[~ex] <= opd[~ex]).all() and (stop[~ex] == 0).all() and (mean[~ex] >= thr).all()
+    assert 0 < ostop.sum() < 40
