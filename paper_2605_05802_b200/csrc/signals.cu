@@ -39,7 +39,6 @@ or_rule_kernel(const double* __restrict__ mean, const int32_t* __restrict__ lens
 // every rollout gets a bit set over those ids, and the Jaccard term of a pair is a few
 // popcounts of AND-ed words instead of K^2 comparisons.  One thread per rollout does
 // the prefix / step-K-action comparisons; thread 0 adds everything up in a fixed order.
-constexpr int kBgSlots = 2048;                  // >= 2 * 32 rollouts * 31 bigrams
 constexpr int kBgWords = 31;                    // 32 * 31 = 992 distinct bigrams at most
 constexpr int kSymPitch = 36;                   // words per staged prefix: 32 + pad, rows 16-byte aligned
 
@@ -300,7 +299,7 @@ int launch_group_signals(const int32_t* seqs, const int32_t* lens, int32_t n_gro
     int threads = (max(pairs_of(N), N * 8) + 31) & ~31;
     if (threads < 64) threads = 64;
     if (threads > 512) threads = 512;
-    int slots = 64;                                  // >= 2 * N * (K - 1) bigrams, at most kBgSlots
+    int slots = 64;                                  // >= 2 * N * (K - 1) bigrams: at most 2048
     while (slots < 2 * N * (K > 1 ? K - 1 : 1)) slots <<= 1;
     int slot_shift = 32;
     while ((1 << (32 - slot_shift)) < slots) --slot_shift;
