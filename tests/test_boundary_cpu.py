@@ -186,3 +186,34 @@ def test_packed_host_entry_rejects_bad_offsets_before_any_launch(lib):
     assert call([0, 5, 9]) == binding.SR_ERR_WORKSPACE            # well-formed, but no arena
     assert call([0], n_groups=0) == binding.SR_OK
     assert lib.sr_gate_host_packed_arena_bytes(4, 8, 64, 64) > lib.sr_gate_host_arena_bytes(4, 8, 64, 64)
+
+
+def test_headers_are_plain_c_and_a_c_program_links(lib, tmp_path):
+    """The boundary is a C ABI: both headers compile as C11 with warnings as errors, and a C
+    program linked against the library reaches the entry points that need no GPU."""
+    import shutil
+    import subprocess
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if cc is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "use_sr_gate.c"
+    src.write_text(
+        '#include <stdio.h>\n#include <string.h>\n#include "sr_gate.h"\n#include "sr_probe.h"\n'
+        "int main(void) {\n"
+        "    if (sr_version() != 100) return 1;\n"
+        "    if (strlen(sr_strerror(SR_ERR_BAD_N)) == 0) return 2;\n"
+        "    /* K <= 32 needs no workspace; the multi-word pipeline says how much it wants */\n"
+        "    if (sr_gate_workspace_bytes(4, 8, 32, 30) != 0) return 3;\n"
+        "    if (sr_gate_workspace_bytes(4, 8, 1024, 1024) == 0) return 4;\n"
+        "    /* argument checks come before any CUDA call: N = 1 is refused on a machine without a GPU too */\n"
+        "    if (sr_gate((const int32_t*)0, (const int32_t*)0, 1, 1, 4, 4, 0.12, SR_NORM_MAXLEN, 0, 0, 0,\n"
+        "                (uint8_t*)0, 0, 0, 0, 0) >= 0) return 5;\n"
+        '    printf("ok %d\\n", sr_version());\n'
+        "    return 0;\n}\n")
+    exe = tmp_path / "use_sr_gate"
+    libdir = os.path.dirname(binding.LIB_PATH)
+    subprocess.run([cc, "-std=c11", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+                    str(src), "-o", str(exe), "-L", libdir, "-lsr_gate", f"-Wl,-rpath,{libdir}"],
+                   check=True, capture_output=True, text=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True, timeout=120)
+    assert out.stdout.strip() == "ok 100"
