@@ -43,6 +43,21 @@ def test_c3_large_group_n16():
     assert 0 < want[3].sum() < 4096
 
 
+@pytest.mark.parametrize("make", ["agent_x128", "large_x16"])
+def test_single_word_batches_of_65536_groups(make):
+    """The single-word kernels on the batch sizes the benchmark's side measurements time
+    (65 536 groups: many groups per CTA, a ragged last CTA): every output of the first and
+    the last groups and of a seeded sample in between, against the oracle."""
+    w = W.agent_gate(K=15, n_groups=65536) if make == "agent_x128" else W.large_group_gate(n_groups=65536)
+    got = gate_gpu(w.seqs, w.lens, w.K, 0.12, w.norm_mode)
+    rng = np.random.default_rng(7)
+    G = w.seqs.shape[0]
+    pick = np.unique(np.concatenate([np.arange(40), np.arange(G - 40, G), rng.integers(0, G, size=600)]))
+    want = oracle.gate(w.seqs[pick], w.lens[pick], w.K, 0.12, w.norm_mode, threads=8)
+    assert_gate_matches(tuple(x[pick] for x in got), want, f"{make}: sampled groups")
+    assert 0 < got[3].sum() < G
+
+
 def test_c4_token_level_small_slice_every_element():
     w = W.token_gate(n_groups=24)
     _check_workload(w, [0.12, 0.6])
