@@ -115,3 +115,27 @@ def test_group_signals_gpu_matches_oracle():
             assert np.array_equal(got[k].view(np.uint64), want[k].view(np.uint64)), (k, K)
         # entropy: device log vs host log, a few ulp per term
         assert np.allclose(got[2], want[2], rtol=0, atol=1e-13)
+
+
+@pytest.mark.gpu
+def test_group_signals_on_65536_groups_of_16():
+    """The batch the kernel's timing is quoted on: first and last groups and a seeded sample
+    against the oracle (bit for bit but for the entropy's logarithms)."""
+    import torch
+    import paper_2605_05802_b200 as sr
+    dev = torch.device("cuda:0")
+    w = W.large_group_gate(n_groups=65536)
+    G = w.seqs.shape[0]
+    outs = [torch.full((G,), -1.0, dtype=torch.float64, device=dev) for _ in range(4)]
+    sr.sr_group_signals(torch.from_numpy(w.seqs).to(dev), torch.from_numpy(w.lens).to(dev), w.K,
+                        unique_prefix_ratio=outs[0], unique_action_ratio=outs[1], action_entropy=outs[2],
+                        bigram_jaccard_mean=outs[3])
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(17)
+    pick = np.unique(np.concatenate([np.arange(32), np.arange(G - 32, G), rng.integers(0, G, size=700)]))
+    want = oracle.group_signals(w.seqs[pick], w.lens[pick], w.K)
+    got = [o.cpu().numpy()[pick] for o in outs]
+    for k in (0, 1, 3):
+        assert np.array_equal(got[k].view(np.uint64), want[k].view(np.uint64)), k
+    assert np.allclose(got[2], want[2], rtol=0, atol=1e-13)
+    assert all((o.cpu().numpy() >= 0).all() for o in outs)        # every group was written
