@@ -95,3 +95,50 @@ def test_decide_on_drawn_shapes(case, G, N, K, stride, vocab, kind, norm):
         lo = ~ex
         assert (stop[lo] == 0).all() and (pd[lo] >= 0).all() and (pd[lo] <= opd[lo]).all(), tag
         assert (mean[lo] <= omean[lo]).all() and (mean[lo] >= thr).all(), tag
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(12))
+def test_single_word_and_incremental_on_drawn_shapes(seed):
+    """Any N in 2..32 and K in 0..32 for the single-word kernels (symbol ids over the whole
+    int32 range); any group size, step limit and termination pattern -- early stops, pauses
+    -- for the incremental gate, which must equal the recomputation after every step."""
+    from helpers import IncrementalGate
+    from paper_2605_05802_b200.binding import SR_NO_ACTION
+    rng = np.random.default_rng(500 + seed)
+    N = int(rng.integers(2, 33))
+    K = int(rng.integers(0, 33))
+    stride = max(4, (K + int(rng.integers(0, 9)) + 3) // 4 * 4)
+    G = int(rng.choice([1, 2, 17, 100, 513, 3000]))
+    vocab = int(rng.choice([1, 2, 3, 17, 300, 2 ** 31 - 1]))
+    kind, norm = int(rng.integers(0, 4)), int(rng.integers(0, 2))
+    seqs, lens = _draw_group_batch(rng, G, N, K, stride, vocab, kind)
+    if seed % 4 == 3:
+        seqs = seqs - (2 ** 31 - 1) // 2                   # negative ids are legal too
+    want = oracle.gate(seqs, lens, K, 0.12, norm, threads=8)
+    thr = float(np.quantile(want[2], rng.random()))
+    want = oracle.gate(seqs, lens, K, thr, norm, threads=8)
+    assert_gate_matches(gate_gpu(seqs, lens, K, thr, norm), want,
+                        f"seed {seed}: N={N} K={K} G={G} vocab={vocab} kind={kind} norm={norm}")
+
+    N = int(rng.choice([2, 3, 5, 8, 8, 13, 16, 32]))
+    steps = int(rng.integers(1, 33))
+    G = int(rng.choice([1, 7, 64, 700]))
+    vocab = int(rng.choice([2, 5, 40, 100000]))
+    norm, thr = int(rng.integers(0, 2)), float(rng.random() * 0.5)
+    inc = IncrementalGate(G, N, steps)
+    base = rng.integers(0, vocab, size=(G, 1, steps))
+    own = rng.integers(0, vocab, size=(G, N, steps))
+    acts = np.where(rng.random((G, N, steps)) < rng.choice([0.05, 0.3, 1.0]), own, base).astype(np.int32)
+    stop_at = rng.integers(0, steps + 1, size=(G, N)) if seed % 2 else np.full((G, N), steps)
+    hist = np.zeros((G, N, 32), dtype=np.int32)
+    hl = np.zeros((G, N), dtype=np.int32)
+    for t in range(steps):
+        act = np.where(t < stop_at, acts[:, :, t], SR_NO_ACTION).astype(np.int32)
+        if seed % 3 == 0:                                  # pauses: a rollout skips a step and resumes
+            act = np.where(rng.random((G, N)) < 0.3, SR_NO_ACTION, act).astype(np.int32)
+        gi, ni = np.nonzero(act != SR_NO_ACTION)
+        hist[gi, ni, hl[gi, ni]] = act[gi, ni]
+        hl[gi, ni] += 1
+        want = oracle.gate(hist, hl, steps, thr, norm, threads=8)
+        assert_gate_matches(inc.step(act, thr, norm), want, f"seed {seed}: incremental N={N} steps={steps} G={G} t={t}")
