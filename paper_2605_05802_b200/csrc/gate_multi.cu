@@ -17,8 +17,8 @@
 //   order    counting sort of the pairs by bin: longest warp tasks first, one team
 //            shape and similar text lengths per bin; warp-task table.
 //   dp       persistent warps pull tasks.  A task is a warp of 32/T teams; a team of
-//            T lanes (T in {1, 2, 4, 8}; up to 32 in small batches) owns one pair, lane l holding R <= 6 consecutive
-//            blocks (32*R rows) in registers.  Lanes are skewed by four columns; the
+//            T lanes (T in {1, 2, 4, 8}; up to 32 in small batches) owns one pair, lane l
+//            holding R <= 6 consecutive blocks (32*R rows) in registers.  Lanes are skewed by four columns; the
 //            delta words of a lane's last block reach the next lane by warp shuffles.
 //            All pairs of a task share (T, R) and have similar lengths, so the warp's
 //            lanes stay busy.
@@ -31,16 +31,18 @@
 // rest), and the threshold caps how large a distance can still matter.  An optimal
 // alignment of distance <= ub never leaves the diagonals d = row - column with
 // |d| + |(m - n) - d| <= ub (Ukkonen's cut-off), so pairs whose bound is small run a
-// banded task, served by CTAs of their own within the dp launch: the pattern's 32-row blocks are grouped in stripes of R blocks, stripe g
-// lives on lane g mod T of a ring of T lanes and is advanced only over the columns where
-// the band crosses it; a stripe the band enters starts from +1 vertical deltas below the
-// stripe above it and a stripe whose upper neighbour the band has left takes +1
-// horizontal deltas from above -- both over-estimates of cells outside the band, which
-// leave every cell on an optimal path exact.  The distance is read from a running score
+// banded task, served by CTAs of their own within the dp launch: the pattern's 32-row
+// blocks are grouped in stripes of R blocks, stripe g lives on lane g mod T of a ring of
+// T lanes and is advanced only over the columns where the band crosses it; a stripe the
+// band enters starts from +1 vertical deltas below the stripe above it and a stripe whose
+// upper neighbour the band has left takes +1 horizontal deltas from above -- both
+// over-estimates of cells outside the band, which leave every cell on an optimal path
+// exact.  The distance is read from a running score
 // at the bottom of the last stripe.  A result within the bound is the exact distance; a
 // result above it only says "more than the bound".  (Banding the exact mode from the
 // mismatch count alone was built as well: 41 % fewer block-columns on the token-level
-// batch, but the banded tasks run at a lower rate and the net gain was a few percent.)
+// batch, but with the banded task bodies next to the six full ones the dp kernel no
+// longer fits the instruction caches and the launch got slower, not faster.)
 //
 // Which rollout of a pair is the pattern is fixed by a round-robin tournament on the
 // indices, so that every pattern CTA of `prep` serves the same number of texts.
