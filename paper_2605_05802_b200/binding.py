@@ -98,13 +98,22 @@ def _check(rc: int) -> None:
         raise SrError(rc, f"sr_gate error {rc}: {msg}")
 
 
-def _ptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype] = None) -> Optional[int]:
+def _ptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype] = None, *, need: Optional[int] = None,
+         host: bool = False, name: str = "tensor") -> Optional[int]:
+    """Address of a caller-owned buffer.  The library dereferences it on the device (on the
+    host for ``host=True``), so a tensor that lives on the wrong side, has another element
+    type, is not contiguous or holds fewer than ``need`` elements is refused here instead of
+    faulting there."""
     if t is None:
         return None
     if dtype is not None and t.dtype != dtype:
-        raise TypeError(f"expected {dtype}, got {t.dtype}")
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
     if not t.is_contiguous():
-        raise ValueError("tensor must be contiguous")
+        raise ValueError(f"{name} must be contiguous")
+    if t.is_cuda == host:
+        raise ValueError(f"{name} must be a {'host' if host else 'CUDA'} tensor")
+    if need is not None and t.numel() < need:
+        raise ValueError(f"{name} holds {t.numel()} elements, the call writes or reads {need}")
     return t.data_ptr()
 
 
@@ -133,10 +142,10 @@ def sr_gate(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, threshold:
     """seqs int32 [G, N, stride] on the device; outputs are preallocated tensors."""
     G, N, stride = seqs.shape
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    _check(load().sr_gate(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
-                          float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
-                          _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
-                          _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(workspace),
+    _check(load().sr_gate(_ptr(seqs, torch.int32), _ptr(lens, torch.int32, need=G * N, name="lens"), G, N, stride, K,
+                          float(threshold), norm_mode, _ptr(pair_dist, torch.int32, need=G * (N * (N - 1) // 2), name="pair_dist"),
+                          _ptr(pair_sum, torch.int32, need=G, name="pair_sum"), _ptr(mean, torch.float64, need=G, name="mean"),
+                          _ptr(stop, torch.uint8, need=G, name="stop"), _ptr(status, torch.int32, need=1, name="status"), _ptr(workspace),
                           ws_bytes, _stream(stream)))
 
 
@@ -153,10 +162,10 @@ def sr_gate_noalloc(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, th
     sr_gate_noalloc_limit_bytes() are refused with SR_ERR_SCRATCH_LIMIT.  Calls that
     may overlap on the device must be serialised by the caller."""
     G, N, stride = seqs.shape
-    _check(load().sr_gate_noalloc(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
-                                  float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
-                                  _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
-                                  _ptr(stop, torch.uint8), _ptr(status, torch.int32),
+    _check(load().sr_gate_noalloc(_ptr(seqs, torch.int32), _ptr(lens, torch.int32, need=G * N, name="lens"), G, N, stride, K,
+                                  float(threshold), norm_mode, _ptr(pair_dist, torch.int32, need=G * (N * (N - 1) // 2), name="pair_dist"),
+                                  _ptr(pair_sum, torch.int32, need=G, name="pair_sum"), _ptr(mean, torch.float64, need=G, name="mean"),
+                                  _ptr(stop, torch.uint8, need=G, name="stop"), _ptr(status, torch.int32, need=1, name="status"),
                                   _stream(stream)))
 
 
@@ -167,11 +176,11 @@ def sr_gate_decide(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, thr
     not computed (exact[g] = 0 marks them, their other outputs are lower bounds)."""
     G, N, stride = seqs.shape
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    _check(load().sr_gate_decide(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
-                                 float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
-                                 _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
-                                 _ptr(stop, torch.uint8), _ptr(exact, torch.uint8),
-                                 _ptr(status, torch.int32), _ptr(workspace), ws_bytes, _stream(stream)))
+    _check(load().sr_gate_decide(_ptr(seqs, torch.int32), _ptr(lens, torch.int32, need=G * N, name="lens"), G, N, stride, K,
+                                 float(threshold), norm_mode, _ptr(pair_dist, torch.int32, need=G * (N * (N - 1) // 2), name="pair_dist"),
+                                 _ptr(pair_sum, torch.int32, need=G, name="pair_sum"), _ptr(mean, torch.float64, need=G, name="mean"),
+                                 _ptr(stop, torch.uint8, need=G, name="stop"), _ptr(exact, torch.uint8, need=G, name="exact"),
+                                 _ptr(status, torch.int32, need=1, name="status"), _ptr(workspace), ws_bytes, _stream(stream)))
 
 
 def sr_gate_stages(seqs, lens, K, threshold, norm_mode=SR_NORM_MAXLEN, *, pair_dist=None, pair_sum=None,
@@ -181,10 +190,10 @@ def sr_gate_stages(seqs, lens, K, threshold, norm_mode=SR_NORM_MAXLEN, *, pair_d
     G, N, stride = seqs.shape
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     handles = (ctypes.c_void_p * 5)(*[e.cuda_event for e in events])
-    _check(load().sr_gate_stages(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
-                                 float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
-                                 _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
-                                 _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(workspace),
+    _check(load().sr_gate_stages(_ptr(seqs, torch.int32), _ptr(lens, torch.int32, need=G * N, name="lens"), G, N, stride, K,
+                                 float(threshold), norm_mode, _ptr(pair_dist, torch.int32, need=G * (N * (N - 1) // 2), name="pair_dist"),
+                                 _ptr(pair_sum, torch.int32, need=G, name="pair_sum"), _ptr(mean, torch.float64, need=G, name="mean"),
+                                 _ptr(stop, torch.uint8, need=G, name="stop"), _ptr(status, torch.int32, need=1, name="status"), _ptr(workspace),
                                  ws_bytes, _stream(stream), handles))
 
 
@@ -202,10 +211,10 @@ def sr_gate_host(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, thres
         if t is not None and t.is_cuda:
             raise ValueError("sr_gate_host takes host tensors")
     G, N, stride = seqs.shape
-    _check(load().sr_gate_host(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
-                               float(threshold), norm_mode, _ptr(pair_dist, torch.int32),
-                               _ptr(pair_sum, torch.int32), _ptr(mean, torch.float64),
-                               _ptr(stop, torch.uint8), _ptr(status, torch.int32), _ptr(arena),
+    _check(load().sr_gate_host(_ptr(seqs, torch.int32, host=True, name="seqs"), _ptr(lens, torch.int32, need=G * N, host=True, name="lens"), G, N, stride, K,
+                               float(threshold), norm_mode, _ptr(pair_dist, torch.int32, need=G * (N * (N - 1) // 2), host=True, name="pair_dist"),
+                               _ptr(pair_sum, torch.int32, need=G, host=True, name="pair_sum"), _ptr(mean, torch.float64, need=G, host=True, name="mean"),
+                               _ptr(stop, torch.uint8, need=G, host=True, name="stop"), _ptr(status, torch.int32, need=1, host=True, name="status"), _ptr(arena),
                                arena.numel() * arena.element_size(), _stream(stream),
                                None if copy_stream is None else copy_stream.cuda_stream))
 
@@ -226,11 +235,12 @@ def sr_gate_host_packed(symbols: torch.Tensor, row_start: torch.Tensor, N: int, 
     rows = row_start.numel() - 1
     if rows < 0 or rows % N:
         raise ValueError("row_start needs n_groups * N + 1 entries")
-    _check(load().sr_gate_host_packed(_ptr(symbols, torch.int32), _ptr(row_start, torch.int64),
+    G = rows // N
+    _check(load().sr_gate_host_packed(_ptr(symbols, torch.int32, host=True, name="symbols"), _ptr(row_start, torch.int64, host=True, name="row_start"),
                                       rows // N, N, stride, K, float(threshold), norm_mode,
-                                      _ptr(pair_dist, torch.int32), _ptr(pair_sum, torch.int32),
-                                      _ptr(mean, torch.float64), _ptr(stop, torch.uint8),
-                                      _ptr(status, torch.int32), _ptr(arena),
+                                      _ptr(pair_dist, torch.int32, need=G * (N * (N - 1) // 2), host=True, name="pair_dist"), _ptr(pair_sum, torch.int32, need=G, host=True, name="pair_sum"),
+                                      _ptr(mean, torch.float64, need=G, host=True, name="mean"), _ptr(stop, torch.uint8, need=G, host=True, name="stop"),
+                                      _ptr(status, torch.int32, need=1, host=True, name="status"), _ptr(arena),
                                       arena.numel() * arena.element_size(), _stream(stream),
                                       None if copy_stream is None else copy_stream.cuda_stream))
 
@@ -249,18 +259,19 @@ def sr_gate_step_incremental(state: torch.Tensor, new_actions: torch.Tensor, thr
                              mean=None, stop=None, status=None, stream=None) -> None:
     G, N = new_actions.shape
     _check(load().sr_gate_step_incremental(
-        _ptr(state), state.numel() * state.element_size(), _ptr(new_actions, torch.int32), G, N,
-        float(threshold), norm_mode, _ptr(pair_dist, torch.int32), _ptr(pair_sum, torch.int32),
-        _ptr(mean, torch.float64), _ptr(stop, torch.uint8), _ptr(status, torch.int32),
+        _ptr(state), state.numel() * state.element_size(), _ptr(new_actions, torch.int32, name="new_actions"), G, N,
+        float(threshold), norm_mode, _ptr(pair_dist, torch.int32, need=G * (N * (N - 1) // 2), name="pair_dist"), _ptr(pair_sum, torch.int32, need=G, name="pair_sum"),
+        _ptr(mean, torch.float64, need=G, name="mean"), _ptr(stop, torch.uint8, need=G, name="stop"), _ptr(status, torch.int32, need=1, name="status"),
         _stream(stream)))
 
 
 def sr_gate_or_rule(mean: torch.Tensor, lens: Optional[torch.Tensor], done: Optional[torch.Tensor],
                     N: int, K: int, threshold: float, tau_high: float, *, tau: Optional[torch.Tensor] = None,
                     stop: torch.Tensor = None, stream=None) -> None:
-    _check(load().sr_gate_or_rule(_ptr(mean, torch.float64), _ptr(lens, torch.int32),
-                                  _ptr(done, torch.uint8), mean.shape[0], N, K, float(threshold),
-                                  float(tau_high), _ptr(tau, torch.float64), _ptr(stop, torch.uint8),
+    G = mean.shape[0]
+    _check(load().sr_gate_or_rule(_ptr(mean, torch.float64), _ptr(lens, torch.int32, need=G * N, name="lens"),
+                                  _ptr(done, torch.uint8, need=G * N, name="done"), mean.shape[0], N, K, float(threshold),
+                                  float(tau_high), _ptr(tau, torch.float64, need=G, name="tau"), _ptr(stop, torch.uint8, need=G, name="stop"),
                                   _stream(stream)))
 
 
@@ -268,19 +279,19 @@ def sr_group_signals(seqs: torch.Tensor, lens: Optional[torch.Tensor], K: int, *
                      unique_prefix_ratio=None, unique_action_ratio=None, action_entropy=None,
                      bigram_jaccard_mean=None, stream=None) -> None:
     G, N, stride = seqs.shape
-    _check(load().sr_group_signals(_ptr(seqs, torch.int32), _ptr(lens, torch.int32), G, N, stride, K,
-                                   _ptr(unique_prefix_ratio, torch.float64),
-                                   _ptr(unique_action_ratio, torch.float64),
-                                   _ptr(action_entropy, torch.float64),
-                                   _ptr(bigram_jaccard_mean, torch.float64), _stream(stream)))
+    _check(load().sr_group_signals(_ptr(seqs, torch.int32), _ptr(lens, torch.int32, need=G * N, name="lens"), G, N, stride, K,
+                                   _ptr(unique_prefix_ratio, torch.float64, need=G, name="unique_prefix_ratio"),
+                                   _ptr(unique_action_ratio, torch.float64, need=G, name="unique_action_ratio"),
+                                   _ptr(action_entropy, torch.float64, need=G, name="action_entropy"),
+                                   _ptr(bigram_jaccard_mean, torch.float64, need=G, name="bigram_jaccard_mean"), _stream(stream)))
 
 
 def sr_batch_stats(adv: torch.Tensor, stop: Optional[torch.Tensor], *, counts: torch.Tensor,
                    sumsq: torch.Tensor, stream=None) -> None:
     """counts: int64 [3] device tensor, sumsq: float64 [2] device tensor (see sr_gate.h)."""
     G, N = adv.shape
-    _check(load().sr_batch_stats(_ptr(adv, torch.float32), _ptr(stop, torch.uint8), G, N,
-                                 _ptr(counts, torch.int64), _ptr(sumsq, torch.float64), _stream(stream)))
+    _check(load().sr_batch_stats(_ptr(adv, torch.float32), _ptr(stop, torch.uint8, need=G, name="stop"), G, N,
+                                 _ptr(counts, torch.int64, need=3, name="counts"), _ptr(sumsq, torch.float64, need=2, name="sumsq"), _stream(stream)))
 
 
 def sr_kept_groups_workspace_bytes(n_groups: int) -> int:
@@ -295,8 +306,8 @@ def sr_kept_groups(stop: Optional[torch.Tensor], zero_var: Optional[torch.Tensor
     if n_groups is None:
         n_groups = (stop if stop is not None else zero_var if zero_var is not None else index).shape[0]
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
-    _check(load().sr_kept_groups(_ptr(stop, torch.uint8), _ptr(zero_var, torch.uint8), n_groups,
-                                 _ptr(index, torch.int32), _ptr(count, torch.int32), _ptr(workspace),
+    _check(load().sr_kept_groups(_ptr(stop, torch.uint8, need=n_groups, name="stop"), _ptr(zero_var, torch.uint8, need=n_groups, name="zero_var"), n_groups,
+                                 _ptr(index, torch.int32, need=n_groups, name="index"), _ptr(count, torch.int32, need=1, name="count"), _ptr(workspace),
                                  ws_bytes, _stream(stream)))
 
 
@@ -311,8 +322,8 @@ def sr_dilution_gain(before: float, after: float) -> float:
 def sr_grpo_advantage(rewards: torch.Tensor, drop_mask: Optional[torch.Tensor], eps: float, *,
                       adv: torch.Tensor, zero_var: Optional[torch.Tensor] = None, stream=None) -> None:
     G, N = rewards.shape
-    _check(load().sr_grpo_advantage(_ptr(rewards, torch.float32), _ptr(drop_mask, torch.uint8), G, N,
-                                    float(eps), _ptr(adv, torch.float32), _ptr(zero_var, torch.uint8),
+    _check(load().sr_grpo_advantage(_ptr(rewards, torch.float32), _ptr(drop_mask, torch.uint8, need=G, name="drop_mask"), G, N,
+                                    float(eps), _ptr(adv, torch.float32, need=G * N, name="adv"), _ptr(zero_var, torch.uint8, need=G, name="zero_var"),
                                     _stream(stream)))
 
 

@@ -217,3 +217,19 @@ def test_headers_are_plain_c_and_a_c_program_links(lib, tmp_path):
                    check=True, capture_output=True, text=True)
     out = subprocess.run([str(exe)], check=True, capture_output=True, text=True, timeout=120)
     assert out.stdout.strip() == "ok 100"
+
+
+def test_binding_refuses_tensors_on_the_wrong_side(lib):
+    """The device entry points dereference their pointers on the GPU: a host tensor handed to
+    them (or a device-style call with the wrong element type) is refused by the binding."""
+    import torch
+    seqs = torch.zeros((2, 8, 16), dtype=torch.int32)
+    stop = torch.zeros(2, dtype=torch.uint8)
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        sr.sr_gate(seqs, None, 15, 0.12, stop=stop)
+    with pytest.raises(TypeError, match="int32"):
+        sr.sr_gate(seqs.to(torch.int64), None, 15, 0.12, stop=stop)
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        sr.sr_grpo_advantage(torch.zeros((2, 8)), None, 1e-6, adv=torch.zeros((2, 8)))
+    with pytest.raises(ValueError, match="contiguous"):
+        sr.sr_gate(seqs.transpose(0, 1), None, 15, 0.12, stop=stop)

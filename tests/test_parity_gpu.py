@@ -475,3 +475,29 @@ def test_advantage_edges():
         r[4, N // 2:] = 0.0
         for eps in (1e-6, 0.0):
             _check_adv(r, None, eps)
+
+
+def test_binding_refuses_short_or_misplaced_buffers():
+    """An output that cannot hold what the call writes, or a host tensor where the library
+    expects device memory, is refused by the binding before anything is launched."""
+    dev = torch.device("cuda:0")
+    w = W.agent_gate(K=15)
+    seqs, lens = torch.from_numpy(w.seqs).to(dev), torch.from_numpy(w.lens).to(dev)
+    G, N, _ = seqs.shape
+    stop = torch.zeros(G, dtype=torch.uint8, device=dev)
+    with pytest.raises(ValueError, match="stop holds"):
+        sr.sr_gate(seqs, lens, w.K, 0.12, stop=stop[: G - 1])
+    with pytest.raises(ValueError, match="pair_dist holds"):
+        sr.sr_gate(seqs, lens, w.K, 0.12, stop=stop, pair_dist=torch.zeros((G, 27), dtype=torch.int32, device=dev))
+    with pytest.raises(ValueError, match="lens holds"):
+        sr.sr_gate(seqs, lens[:-1], w.K, 0.12, stop=stop)
+    with pytest.raises(ValueError, match="CUDA tensor"):
+        sr.sr_gate(seqs, lens.cpu(), w.K, 0.12, stop=stop)
+    with pytest.raises(ValueError, match="host tensor"):
+        sr.sr_gate_host(seqs, None, w.K, 0.12, stop=stop.cpu(), arena=torch.empty(1 << 20, dtype=torch.uint8, device=dev))
+    rewards = torch.rand((G, N), device=dev)
+    with pytest.raises(ValueError, match="adv holds"):
+        sr.sr_grpo_advantage(rewards, None, 1e-6, adv=torch.empty((G, N - 1), device=dev))
+    sr.sr_gate(seqs, lens, w.K, 0.12, stop=stop)                       # and the well-formed call still runs
+    torch.cuda.synchronize()
+    assert np.array_equal(stop.cpu().numpy(), oracle.gate(w.seqs, w.lens, w.K, 0.12)[3])
